@@ -1,0 +1,163 @@
+/*
+ * fp8mlp — FP8 Smooth-SwiGLU MLP block (forward + backward) for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of libfp8mlp.so.  The block is the Llama-style MLP
+ *     Y = (Swish(x W2) * (x W1)) W3
+ * trained in FP8 as in "Scaling FP8 training to trillion-token LLMs": E4M3 operands in the
+ * forward phase, E5M2 gradients in the backward phase, per-tensor scales taken from amax
+ * buffers, and the paper's Smooth-SwiGLU (Section 4.4, Eq. 2): a per-channel scale s_i is
+ * applied to the SwiGLU output before it is quantised and s_i^-1 is folded into row i of W3
+ * before W3 is quantised.  Naming follows the paper (Section 4.1): W1 is the linear branch,
+ * W2 the Swish (gate) branch, W3 the last linear layer.  T = tokens, d = d_model, f = d_ff.
+ *
+ * Conventions for every entry point
+ *   - All tensor / amax / scale pointers are DEVICE pointers owned by the caller, row-major,
+ *     16-byte aligned; the library never frees or reallocates them.  d and f must be
+ *     multiples of 16 (FP8MLP_ERR_SHAPE otherwise); T is any value >= 0 and <= T_max.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work on it and return; nothing synchronises the device.
+ *   - The return value is FP8MLP_OK (0) or a negative FP8MLP_ERR_* code.  Argument errors are
+ *     detected before anything is launched.  Nothing throws or aborts across this boundary.
+ *   - bf16 tensors are passed as void* (2 bytes per element); FP8 codes as uint8_t.
+ *   - Rounding: FP8 casts are round-to-nearest-even and saturate to the largest finite value
+ *     (448 for E4M3, 57344 for E5M2); bf16 outputs are round-to-nearest-even from fp32.
+ */
+#ifndef FP8MLP_H_
+#define FP8MLP_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define FP8MLP_API __attribute__((visibility("default")))
+#else
+#define FP8MLP_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fp8mlp_ctx fp8mlp_ctx; /* opaque: owns the FP8 operand copies, saved activations, status word */
+
+enum {
+    FP8MLP_OK = 0,
+    FP8MLP_ERR_ARG = -1,     /* null pointer / bad enum value                                   */
+    FP8MLP_ERR_SHAPE = -2,   /* negative size, d or f not a multiple of 16, T > T_max           */
+    FP8MLP_ERR_ALIGN = -3,   /* a tensor pointer is not 16-byte aligned                         */
+    FP8MLP_ERR_CUDA = -4,    /* a CUDA runtime/driver call failed (see fp8mlp_last_cuda_error)  */
+    FP8MLP_ERR_TIMEOUT = -5, /* a kernel gave up on a bounded wait (device status word)         */
+    FP8MLP_ERR_STATE = -6    /* backward without a matching forward that saved activations      */
+};
+enum { FP8MLP_E4M3 = 0, FP8MLP_E5M2 = 1 };
+enum { FP8MLP_BF16 = 0, FP8MLP_F32 = 1 };
+enum {
+    FP8MLP_SMOOTH = 1,       /* per-channel Smooth-SwiGLU scales; without it one per-tensor scale for H */
+    FP8MLP_SAVE_FOR_BWD = 2  /* forward keeps bf16 G = x W2 and U = x W1 for backward               */
+};
+enum {
+    FP8MLP_SCALE_GIVEN = 0,              /* delayed scaling: use the scale buffers as they are  */
+    FP8MLP_SCALE_FROM_CURRENT_AMAX = 1   /* just-in-time: derive every scale from this call's data */
+};
+enum { /* fp8mlp_workspace: internal buffers, for inspection by tests */
+    FP8MLP_WS_XQ = 0,   /* E4M3 [T,d]   quantised x                                   */
+    FP8MLP_WS_W12Q = 1, /* E4M3 [d,2f]  quantised [W2 | W1]: gate columns [0,f), linear [f,2f) */
+    FP8MLP_WS_W3Q = 2,  /* E4M3 [f,d]   quantised diag(s^-1) W3                        */
+    FP8MLP_WS_HQ = 3,   /* E4M3 [T,f]   Q(s_i * SwiGLU)                                */
+    FP8MLP_WS_GU = 4,   /* bf16 [T,2f]  saved G | U                                    */
+    FP8MLP_WS_DYQ = 5,  /* E5M2 [T,d]   quantised dY                                   */
+    FP8MLP_WS_DZQ = 6   /* E5M2 [T,2f]  quantised [dG | dU]                            */
+};
+
+/* The paper's scaling state (Section 2: per-tensor scaling, delayed or just-in-time; Section 4.4:
+ * per-channel s_i).  Every member is a device pointer to float(s), caller-owned; the library
+ * keeps no history.  A scale multiplies the tensor before the cast: code = Q(v * scale).
+ *   scales.h[f]: Smooth on  -> s_i, powers of two;  Smooth off -> the per-tensor scale, repeated.
+ *   amax.h[f]  : per-channel max |SwiGLU output| before scaling (Section 4.4, steps 1-2).
+ *   amax.w3    : max |W3[i,j] / s_i|  (the tensor that is actually quantised).
+ *   w12 / dz   : one scale for the concatenated [W2|W1] and [dG|dU] operands; amax of W1 and
+ *                W2 are still reported separately. */
+typedef struct { float *x, *w12, *w3, *dy, *dz, *h; } fp8mlp_scales;
+typedef struct { float *x, *w1, *w2, *w3, *dy, *dz, *h; } fp8mlp_amax;
+
+/* Creates a context for T <= T_max tokens.  Allocates its workspace on the current device
+ * (about T_max*(2d + 7f) + 3*d*f bytes).  Host call; may synchronise. */
+FP8MLP_API int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d_model, int64_t d_ff, uint32_t flags);
+FP8MLP_API int fp8mlp_destroy(fp8mlp_ctx* ctx);
+FP8MLP_API const char* fp8mlp_strerror(int code);
+/* Text of the last CUDA error this thread's calls ran into ("" if none). */
+FP8MLP_API const char* fp8mlp_last_cuda_error(void);
+/* Synchronises `stream`, then returns FP8MLP_ERR_TIMEOUT if any kernel of this context gave up on
+ * a bounded wait since the last call (and clears the word), else FP8MLP_OK. */
+FP8MLP_API int fp8mlp_status(fp8mlp_ctx* ctx, void* stream);
+/* Device pointer and size in bytes of one of the FP8MLP_WS_* buffers (sized for T_max). */
+FP8MLP_API int fp8mlp_workspace(fp8mlp_ctx* ctx, int which, void** ptr, int64_t* bytes);
+/* Number of kernels this library has launched in this process so far (all contexts). */
+FP8MLP_API int64_t fp8mlp_launch_count(void);
+
+/* Per-tensor quantisation (Section 2: "scaling each tensor individually based on its specific
+ * range of values"; Section 4.4 for row_mul).
+ *   dst[r, c] = Q_fmt( (src[r, c] * row_mul[r]) * scale ),  r < rows, c < cols
+ *   src       rows x cols, src_dtype FP8MLP_BF16 or FP8MLP_F32, contiguous.
+ *   dst       FP8 codes, leading dimension ld_dst >= cols (bytes), ld_dst % 16 == 0.
+ *   row_mul   nullable; per-row multiplier (s_i^-1 for W3' = diag(s^-1) W3).
+ *   scale     device float.  SCALE_GIVEN: read.  SCALE_FROM_CURRENT_AMAX: written first, as
+ *             fmt_max / amax (1 if amax is 0 or not finite), then used; costs a second pass
+ *             over src.
+ *   amax      device float, receives max |src * row_mul|.  Nullable in SCALE_GIVEN mode,
+ *             required in SCALE_FROM_CURRENT_AMAX mode.
+ * cols % 16 == 0.  rows == 0 is allowed (amax becomes 0). */
+FP8MLP_API int fp8mlp_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, int fp8_fmt,
+                    int scale_mode, float* scale, float* amax, const float* row_mul,
+                    uint8_t* dst, int64_t ld_dst, void* stream);
+
+/* amax -> scale bookkeeping between steps (Section 2, delayed scaling; Section 4.4 step 3).
+ *   x, w3, dy : scale = fmt_max / amax.     w12 : 448 / max(amax.w1, amax.w2).
+ *   h[i]      : Smooth on: largest power of two p with p * amax.h[i] <= 448; off: 448 / max_i amax.h[i].
+ *   dz        : largest power of two p with p * amax.dz <= 57344.
+ * A zero or non-finite amax gives scale 1.  Members of `amax` that are NULL are skipped together
+ * with their scale. */
+FP8MLP_API int fp8mlp_update_scales(fp8mlp_ctx* ctx, const fp8mlp_amax* amax, fp8mlp_scales* scales, void* stream);
+
+/* Forward (Eq. 2 and the merge of Section 4.4; Section 6.2 for the operand formats).
+ *   x_bf16 [T,d]; W1, W2 [d,f], W3 [f,d] fp32 master weights; y_bf16 [T,d] output.
+ *   1. Xq = Q(x sx); [W2q|W1q] = Q(W sw12); G = Xq W2q / (sx sw12), U likewise (fp32 accumulate)
+ *   2. H = U * G * sigma(G); amax.h[i] = max_t |H[t,i]|; Hq = Q(H * s_i)   (never stored unquantised)
+ *   3. W3q = Q((W3[i,:] / s_i) sw3)  (Smooth off: Q(W3 sw3));  Y = Hq W3q / sw3  (Smooth off: / (sw3 sh))
+ *   SCALE_GIVEN: `scales` are read; `amax` (nullable, members nullable) receives this call's maxima.
+ *   SCALE_FROM_CURRENT_AMAX: both structs must be complete; scales.x/w12/h/w3 are overwritten from
+ *   this call's data first (runs step 1-2 twice: once for the per-channel maxima, once for the codes).
+ *   With FP8MLP_SAVE_FOR_BWD in the context flags, bf16 G and U are kept for fp8mlp_backward. */
+FP8MLP_API int fp8mlp_forward(fp8mlp_ctx* ctx, int64_t T, const void* x_bf16,
+                   const float* W1, const float* W2, const float* W3,
+                   int scale_mode, fp8mlp_scales* scales, fp8mlp_amax* amax,
+                   void* y_bf16, void* stream);
+
+/* Backward (Section 6.2: E5M2 gradients; proof of Theorem 1 for the gate derivative
+ * sigma(g) + g sigma'(g)).  Needs the preceding fp8mlp_forward on the same context, same T, with
+ * FP8MLP_SAVE_FOR_BWD (FP8MLP_ERR_STATE otherwise); uses the same `scales` the forward used.
+ *   dYq = Q_e5m2(dY sdy);  dH = s (.) (dYq W3q^T) / (sdy sw3)  (Smooth off: no s)
+ *   dU = dH * G sigma(G);  dG = dH * U * sigma(G) (1 + G (1 - sigma(G)));  dZq = Q_e5m2([dG|dU] sdz)
+ *   dX = dZq [W2q|W1q]^T / (sdz sw12)  -> bf16 [T,d]
+ *   [dW2|dW1] = Xq^T dZq / (sx sdz)    -> fp32 [d,f] each, overwritten
+ *   dW3[i,:] = (Hq^T dYq)[i,:] / (sdy s_i) -> fp32 [f,d], overwritten
+ * Every Q is straight-through and s is a constant.  scale_mode as in forward, for dy and dz. */
+FP8MLP_API int fp8mlp_backward(fp8mlp_ctx* ctx, int64_t T, const void* dy_bf16,
+                    int scale_mode, fp8mlp_scales* scales, fp8mlp_amax* amax,
+                    void* dx_bf16, float* dW1, float* dW2, float* dW3, void* stream);
+
+/* One FP8 GEMM of the kind the block is made of, exposed for tests and tuning (Section 6.2:
+ * quantised operands, high-precision accumulation and output).
+ *   out[m, n] = (sum_k A(m,k) B(n,k)) * ((1 / *scale_a) * (1 / *scale_b)),  fp32 accumulate,
+ *   out fp32 [M,N] row-major.  scale_a / scale_b: device floats, nullable (= 1).
+ *   a_kmajor != 0: A is stored [M,K] (K contiguous); == 0: stored [K,M] (M contiguous).
+ *   b_kmajor != 0: B is stored [N,K];                == 0: stored [K,N].
+ *   a_fmt / b_fmt: FP8MLP_E4M3 or FP8MLP_E5M2.  M, N, K multiples of 16 and > 0. */
+FP8MLP_API int fp8mlp_gemm_fp8(int64_t M, int64_t N, int64_t K,
+                    const uint8_t* A, int a_kmajor, int a_fmt,
+                    const uint8_t* B, int b_kmajor, int b_fmt,
+                    const float* scale_a, const float* scale_b, float* out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP8MLP_H_ */

@@ -1,0 +1,400 @@
+// C ABI of libfp8mlp (declared in include/fp8mlp.h): argument validation, the context's
+// workspace, and the sequence of kernels that makes up forward and backward.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "gemm.cuh"
+#include "quantize.cuh"
+
+namespace fp8mlp {
+
+namespace {
+thread_local char g_last_error[512] = "";
+std::atomic<int64_t> g_launches{0};
+}  // namespace
+
+void set_cuda_error(const char* what, cudaError_t e) {
+    std::snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
+}
+void set_cuda_error_str(const char* what, const char* msg) {
+    std::snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, msg);
+}
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+// Sets up to 8 device floats to zero in one launch (amax accumulators).
+struct ZeroList { float* p[8]; };
+__global__ void zero_floats_kernel(ZeroList z) {
+    if (threadIdx.x < 8 && z.p[threadIdx.x] != nullptr) *z.p[threadIdx.x] = 0.0f;
+}
+
+}  // namespace fp8mlp
+
+using namespace fp8mlp;
+
+struct fp8mlp_ctx {
+    int64_t T_max, d, f;
+    uint32_t flags;
+    int device, sm_count;
+    uint8_t *xq, *w12q, *w3q, *hq, *dyq, *dzq;
+    uint16_t* gu;
+    float* inv_s;     // [f] 1 / s_h: row multipliers of W3' = diag(s^-1) W3
+    float* dummy;     // [8 + f] sinks for amax outputs the caller did not ask for
+    int* status;      // bounded-wait status word
+    int64_t saved_T;  // tokens of the last forward that saved activations, -1 if none
+    int64_t bytes[7];
+};
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int zero_floats(std::initializer_list<float*> ptrs, cudaStream_t st) {
+    ZeroList z{};
+    int n = 0;
+    for (float* p : ptrs) z.p[n++] = p;
+    zero_floats_kernel<<<1, 32, 0, st>>>(z);
+    FP8MLP_LAUNCH_CHECK();
+    return FP8MLP_OK;
+}
+
+#define FP8MLP_TRY(expr)                    \
+    do {                                    \
+        int rc__ = (expr);                  \
+        if (rc__ != FP8MLP_OK) return rc__; \
+    } while (0)
+
+// amax (optional) + cast of one tensor, in either scale mode.  amax must be non-null.
+int quantize_tensor(const void* src, int dtype, int64_t rows, int64_t cols, int fmt, int mode, float* scale,
+                    float* amax, const float* amax_other, const float* row_mul, uint8_t* dst, int64_t ld_dst,
+                    int sm_count, cudaStream_t st) {
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
+        FP8MLP_TRY(run_quantize_pass(false, true, src, dtype, rows, cols, fmt, row_mul, nullptr, nullptr, 0, amax, sm_count, st));
+        FP8MLP_TRY(run_scale_from_amax(fmt, amax, amax_other, scale, st));
+        return run_quantize_pass(true, false, src, dtype, rows, cols, fmt, row_mul, scale, dst, ld_dst, nullptr, sm_count, st);
+    }
+    return run_quantize_pass(true, true, src, dtype, rows, cols, fmt, row_mul, scale, dst, ld_dst, amax, sm_count, st);
+}
+
+GemmArgs base_args(fp8mlp_ctx* c, int M, int N, int K) {
+    GemmArgs a{};
+    a.M = M; a.N = N; a.K = K;
+    a.n_tile_cols = kBlockN;
+    a.b1_offset = 128;
+    a.group_m = 16;
+    a.status = c ? c->status : nullptr;
+    a.n_split = N;
+    a.ld_out = N;
+    a.store = 1;
+    return a;
+}
+
+// G|U = Xq [W2q|W1q] with the SwiGLU / Smooth-SwiGLU epilogue
+int gemm1_swiglu(fp8mlp_ctx* c, int64_t T, const fp8mlp_scales* s, float* amax_h, int store, cudaStream_t st) {
+    CUtensorMap tmA, tmB0, tmB1;
+    FP8MLP_TRY(make_tmap_u8(&tmA, c->xq, c->d, T, c->d));
+    FP8MLP_TRY(make_tmap_u8(&tmB0, c->w12q, c->f, c->d, 2 * c->f));
+    FP8MLP_TRY(make_tmap_u8(&tmB1, c->w12q + c->f, c->f, c->d, 2 * c->f));
+    GemmArgs a = base_args(c, static_cast<int>(T), static_cast<int>(c->f), static_cast<int>(c->d));
+    a.n_tile_cols = 128;
+    a.b1_offset = 0;
+    a.s0 = s->x; a.s1 = s->w12;
+    a.s_h = s->h;
+    a.store = store;
+    a.hq = c->hq;
+    a.gu = (c->flags & FP8MLP_SAVE_FOR_BWD) ? c->gu : nullptr;
+    a.amax_h = reinterpret_cast<unsigned int*>(amax_h);
+    return launch_gemm(EPI_SWIGLU_FWD, false, true, FP8MLP_E4M3, FP8MLP_E4M3, tmA, tmB0, tmB1, a, c->sm_count, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fp8mlp_strerror(int code) {
+    switch (code) {
+        case FP8MLP_OK: return "ok";
+        case FP8MLP_ERR_ARG: return "invalid argument (null pointer or bad enum value)";
+        case FP8MLP_ERR_SHAPE: return "invalid shape (negative, not a multiple of 16, or T > T_max)";
+        case FP8MLP_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case FP8MLP_ERR_CUDA: return "CUDA call failed";
+        case FP8MLP_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
+        case FP8MLP_ERR_STATE: return "backward without a matching forward that saved activations";
+        default: return "unknown error code";
+    }
+}
+
+const char* fp8mlp_last_cuda_error(void) { return g_last_error; }
+
+int64_t fp8mlp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_t flags) {
+    if (out == nullptr) return FP8MLP_ERR_ARG;
+    *out = nullptr;
+    if (flags & ~uint32_t(FP8MLP_SMOOTH | FP8MLP_SAVE_FOR_BWD)) return FP8MLP_ERR_ARG;
+    if (T_max < 0 || d <= 0 || f <= 0 || d % 16 != 0 || f % 16 != 0) return FP8MLP_ERR_SHAPE;
+    if (T_max > (1 << 30) || d > (1 << 24) || f > (1 << 24)) return FP8MLP_ERR_SHAPE;
+    fp8mlp_ctx* c = new (std::nothrow) fp8mlp_ctx();
+    if (c == nullptr) return FP8MLP_ERR_ARG;
+    std::memset(c, 0, sizeof(*c));
+    c->T_max = T_max; c->d = d; c->f = f; c->flags = flags; c->saved_T = -1;
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    const int64_t Tm = T_max > 0 ? T_max : 1;
+    c->bytes[FP8MLP_WS_XQ] = Tm * d;
+    c->bytes[FP8MLP_WS_W12Q] = d * 2 * f;
+    c->bytes[FP8MLP_WS_W3Q] = f * d;
+    c->bytes[FP8MLP_WS_HQ] = Tm * f;
+    c->bytes[FP8MLP_WS_GU] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * 2 * f * 2 : 16;
+    c->bytes[FP8MLP_WS_DYQ] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * d : 16;
+    c->bytes[FP8MLP_WS_DZQ] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * 2 * f : 16;
+    void** slots[7] = {(void**)&c->xq, (void**)&c->w12q, (void**)&c->w3q, (void**)&c->hq,
+                       (void**)&c->gu, (void**)&c->dyq, (void**)&c->dzq};
+    for (int i = 0; i < 7 && e == cudaSuccess; ++i) e = cudaMalloc(slots[i], static_cast<size_t>(c->bytes[i]));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&c->inv_s, sizeof(float) * f);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&c->dummy, sizeof(float) * (8 + f));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&c->status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int));
+    if (e != cudaSuccess) {
+        set_cuda_error("fp8mlp_create", e);
+        fp8mlp_destroy(c);
+        return FP8MLP_ERR_CUDA;
+    }
+    *out = c;
+    return FP8MLP_OK;
+}
+
+int fp8mlp_destroy(fp8mlp_ctx* c) {
+    if (c == nullptr) return FP8MLP_OK;
+    void* ptrs[] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq, c->inv_s, c->dummy, c->status};
+    for (void* p : ptrs)
+        if (p != nullptr) cudaFree(p);
+    delete c;
+    return FP8MLP_OK;
+}
+
+int fp8mlp_status(fp8mlp_ctx* c, void* stream) {
+    if (c == nullptr) return FP8MLP_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int word = 0;
+    FP8MLP_CUDA_CHECK(cudaMemcpyAsync(&word, c->status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    FP8MLP_CUDA_CHECK(cudaStreamSynchronize(st));
+    if (word != STATUS_OK) {
+        FP8MLP_CUDA_CHECK(cudaMemsetAsync(c->status, 0, sizeof(int), st));
+        return FP8MLP_ERR_TIMEOUT;
+    }
+    return FP8MLP_OK;
+}
+
+int fp8mlp_workspace(fp8mlp_ctx* c, int which, void** ptr, int64_t* bytes) {
+    if (c == nullptr || ptr == nullptr || bytes == nullptr || which < 0 || which > FP8MLP_WS_DZQ) return FP8MLP_ERR_ARG;
+    void* all[7] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq};
+    *ptr = all[which];
+    *bytes = c->bytes[which];
+    return FP8MLP_OK;
+}
+
+int fp8mlp_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, int fp8_fmt, int scale_mode,
+                    float* scale, float* amax, const float* row_mul, uint8_t* dst, int64_t ld_dst, void* stream) {
+    if (src == nullptr || dst == nullptr || scale == nullptr) return FP8MLP_ERR_ARG;
+    if (src_dtype != FP8MLP_BF16 && src_dtype != FP8MLP_F32) return FP8MLP_ERR_ARG;
+    if (fp8_fmt != FP8MLP_E4M3 && fp8_fmt != FP8MLP_E5M2) return FP8MLP_ERR_ARG;
+    if (scale_mode != FP8MLP_SCALE_GIVEN && scale_mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
+    if (scale_mode == FP8MLP_SCALE_FROM_CURRENT_AMAX && amax == nullptr) return FP8MLP_ERR_ARG;
+    if (rows < 0 || cols < 0 || cols % 16 != 0 || ld_dst < cols || ld_dst % 16 != 0) return FP8MLP_ERR_SHAPE;
+    if (!aligned16(src) || !aligned16(dst)) return FP8MLP_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev = 0, sms = 0;
+    FP8MLP_CUDA_CHECK(cudaGetDevice(&dev));
+    FP8MLP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (amax != nullptr) FP8MLP_TRY(zero_floats({amax}, st));
+    if (scale_mode == FP8MLP_SCALE_FROM_CURRENT_AMAX)
+        return quantize_tensor(src, src_dtype, rows, cols, fp8_fmt, scale_mode, scale, amax, nullptr, row_mul, dst,
+                               ld_dst, sms, st);
+    return run_quantize_pass(true, amax != nullptr, src, src_dtype, rows, cols, fp8_fmt, row_mul, scale, dst, ld_dst,
+                             amax, sms, st);
+}
+
+int fp8mlp_update_scales(fp8mlp_ctx* c, const fp8mlp_amax* am, fp8mlp_scales* sc, void* stream) {
+    if (c == nullptr || am == nullptr || sc == nullptr) return FP8MLP_ERR_ARG;
+    UpdateScalesArgs a{};
+    a.amax_x = am->x; a.amax_w1 = am->w1; a.amax_w2 = am->w2; a.amax_w3 = am->w3;
+    a.amax_dy = am->dy; a.amax_dz = am->dz; a.amax_h = am->h;
+    a.scale_x = sc->x; a.scale_w12 = sc->w12; a.scale_w3 = sc->w3;
+    a.scale_dy = sc->dy; a.scale_dz = sc->dz; a.scale_h = sc->h;
+    a.f = c->f;
+    a.smooth = (c->flags & FP8MLP_SMOOTH) ? 1 : 0;
+    return run_update_scales(a, c->sm_count, static_cast<cudaStream_t>(stream));
+}
+
+int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, const float* W2, const float* W3,
+                   int mode, fp8mlp_scales* sc, fp8mlp_amax* am, void* y, void* stream) {
+    if (c == nullptr || sc == nullptr || W1 == nullptr || W2 == nullptr || W3 == nullptr) return FP8MLP_ERR_ARG;
+    if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
+    if (T < 0 || T > c->T_max) return FP8MLP_ERR_SHAPE;
+    if (T > 0 && (x == nullptr || y == nullptr)) return FP8MLP_ERR_ARG;
+    if (sc->x == nullptr || sc->w12 == nullptr || sc->w3 == nullptr || sc->h == nullptr) return FP8MLP_ERR_ARG;
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX &&
+        (am == nullptr || am->x == nullptr || am->w1 == nullptr || am->w2 == nullptr || am->w3 == nullptr || am->h == nullptr))
+        return FP8MLP_ERR_ARG;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(W1) || !aligned16(W2) || !aligned16(W3)) return FP8MLP_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool smooth = (c->flags & FP8MLP_SMOOTH) != 0;
+    const int64_t d = c->d, f = c->f;
+    // amax sinks the caller did not provide
+    float* a_x = (am && am->x) ? am->x : c->dummy + 0;
+    float* a_w1 = (am && am->w1) ? am->w1 : c->dummy + 1;
+    float* a_w2 = (am && am->w2) ? am->w2 : c->dummy + 2;
+    float* a_w3 = (am && am->w3) ? am->w3 : c->dummy + 3;
+    float* a_h = (am && am->h) ? am->h : c->dummy + 8;
+    c->saved_T = -1;
+
+    FP8MLP_TRY(zero_floats({a_x, a_w1, a_w2, a_w3}, st));
+    FP8MLP_CUDA_CHECK(cudaMemsetAsync(a_h, 0, sizeof(float) * f, st));
+
+    // x -> E4M3
+    FP8MLP_TRY(quantize_tensor(x, FP8MLP_BF16, T, d, FP8MLP_E4M3, mode, sc->x, a_x, nullptr, nullptr, c->xq, d, c->sm_count, st));
+    // [W2 | W1] -> E4M3 with one scale
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
+        FP8MLP_TRY(run_quantize_pass(false, true, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, nullptr, nullptr, 0, a_w1, c->sm_count, st));
+        FP8MLP_TRY(run_quantize_pass(false, true, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, nullptr, nullptr, 0, a_w2, c->sm_count, st));
+        FP8MLP_TRY(run_scale_from_amax(FP8MLP_E4M3, a_w1, a_w2, sc->w12, st));
+        FP8MLP_TRY(run_quantize_pass(true, false, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, sc->w12, c->w12q, 2 * f, nullptr, c->sm_count, st));
+        FP8MLP_TRY(run_quantize_pass(true, false, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, sc->w12, c->w12q + f, 2 * f, nullptr, c->sm_count, st));
+    } else {
+        FP8MLP_TRY(run_quantize_pass(true, true, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, sc->w12, c->w12q, 2 * f, a_w2, c->sm_count, st));
+        FP8MLP_TRY(run_quantize_pass(true, true, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, sc->w12, c->w12q + f, 2 * f, a_w1, c->sm_count, st));
+    }
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
+        // calibration pass: per-channel maxima of H, then s_i (or the per-tensor scale)
+        if (T > 0) FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/0, st));
+        UpdateScalesArgs u{};
+        u.amax_h = a_h; u.scale_h = sc->h; u.f = f; u.smooth = smooth ? 1 : 0;
+        FP8MLP_TRY(run_update_scales(u, c->sm_count, st));
+    }
+    // W3' = diag(1/s) W3 -> E4M3
+    const float* row_mul = nullptr;
+    if (smooth) {
+        FP8MLP_TRY(run_reciprocal(sc->h, c->inv_s, f, st));
+        row_mul = c->inv_s;
+    }
+    FP8MLP_TRY(quantize_tensor(W3, FP8MLP_F32, f, d, FP8MLP_E4M3, mode, sc->w3, a_w3, nullptr, row_mul, c->w3q, d, c->sm_count, st));
+    if (T == 0) { c->saved_T = (c->flags & FP8MLP_SAVE_FOR_BWD) ? 0 : -1; return FP8MLP_OK; }
+
+    FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/1, st));
+
+    // Y = Hq W3q
+    CUtensorMap tmA, tmB;
+    FP8MLP_TRY(make_tmap_u8(&tmA, c->hq, f, T, f));
+    FP8MLP_TRY(make_tmap_u8(&tmB, c->w3q, d, f, d));
+    GemmArgs a = base_args(c, static_cast<int>(T), static_cast<int>(d), static_cast<int>(f));
+    a.s0 = sc->w3;
+    a.s1 = smooth ? nullptr : sc->h;
+    a.out_bf16 = static_cast<uint16_t*>(y);
+    FP8MLP_TRY(launch_gemm(EPI_BF16, false, true, FP8MLP_E4M3, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
+    if (c->flags & FP8MLP_SAVE_FOR_BWD) c->saved_T = T;
+    return FP8MLP_OK;
+}
+
+int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_scales* sc, fp8mlp_amax* am,
+                    void* dx, float* dW1, float* dW2, float* dW3, void* stream) {
+    if (c == nullptr || sc == nullptr || dW1 == nullptr || dW2 == nullptr || dW3 == nullptr) return FP8MLP_ERR_ARG;
+    if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
+    if (T < 0 || T > c->T_max) return FP8MLP_ERR_SHAPE;
+    if (!(c->flags & FP8MLP_SAVE_FOR_BWD) || c->saved_T != T) return FP8MLP_ERR_STATE;
+    if (T > 0 && (dy == nullptr || dx == nullptr)) return FP8MLP_ERR_ARG;
+    if (sc->x == nullptr || sc->w12 == nullptr || sc->w3 == nullptr || sc->h == nullptr || sc->dy == nullptr || sc->dz == nullptr)
+        return FP8MLP_ERR_ARG;
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX && (am == nullptr || am->dy == nullptr || am->dz == nullptr)) return FP8MLP_ERR_ARG;
+    if (!aligned16(dy) || !aligned16(dx) || !aligned16(dW1) || !aligned16(dW2) || !aligned16(dW3)) return FP8MLP_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool smooth = (c->flags & FP8MLP_SMOOTH) != 0;
+    const int64_t d = c->d, f = c->f;
+    float* a_dy = (am && am->dy) ? am->dy : c->dummy + 4;
+    float* a_dz = (am && am->dz) ? am->dz : c->dummy + 5;
+    FP8MLP_TRY(zero_floats({a_dy, a_dz}, st));
+    if (T == 0) {   // empty batch: the weight gradients are sums over no tokens
+        FP8MLP_CUDA_CHECK(cudaMemsetAsync(dW1, 0, sizeof(float) * d * f, st));
+        FP8MLP_CUDA_CHECK(cudaMemsetAsync(dW2, 0, sizeof(float) * d * f, st));
+        FP8MLP_CUDA_CHECK(cudaMemsetAsync(dW3, 0, sizeof(float) * d * f, st));
+        return FP8MLP_OK;
+    }
+    const int Ti = static_cast<int>(T), di = static_cast<int>(d), fi = static_cast<int>(f);
+
+    // dY -> E5M2
+    FP8MLP_TRY(quantize_tensor(dy, FP8MLP_BF16, T, d, FP8MLP_E5M2, mode, sc->dy, a_dy, nullptr, nullptr, c->dyq, d, c->sm_count, st));
+
+    // dH~ = dYq W3q^T with the SwiGLU-backward epilogue -> dZq = [dG | dU]
+    {
+        CUtensorMap tmA, tmB;
+        FP8MLP_TRY(make_tmap_u8(&tmA, c->dyq, d, T, d));
+        FP8MLP_TRY(make_tmap_u8(&tmB, c->w3q, d, f, d));
+        GemmArgs a = base_args(c, Ti, fi, di);
+        a.s0 = sc->dy; a.s1 = sc->w3;
+        a.s_h = sc->h; a.smooth = smooth ? 1 : 0;
+        a.gu = c->gu; a.sdz = sc->dz; a.dzq = c->dzq;
+        a.amax_dz = reinterpret_cast<unsigned int*>(a_dz);
+        if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
+            a.store = 0;
+            FP8MLP_TRY(launch_gemm(EPI_SWIGLU_BWD, false, false, FP8MLP_E5M2, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
+            UpdateScalesArgs u{};
+            u.amax_dz = a_dz; u.scale_dz = sc->dz;
+            FP8MLP_TRY(run_update_scales(u, c->sm_count, st));
+            a.store = 1;
+        }
+        FP8MLP_TRY(launch_gemm(EPI_SWIGLU_BWD, false, false, FP8MLP_E5M2, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
+    }
+    // dW3 = diag(1/s) (Hq^T dYq)
+    {
+        CUtensorMap tmA, tmB;
+        FP8MLP_TRY(make_tmap_u8(&tmA, c->hq, f, T, f));
+        FP8MLP_TRY(make_tmap_u8(&tmB, c->dyq, d, T, d));
+        GemmArgs a = base_args(c, fi, di, Ti);
+        a.s0 = sc->dy; a.row_s = sc->h;
+        a.out_f32_0 = dW3; a.out_f32_1 = dW3;
+        FP8MLP_TRY(launch_gemm(EPI_F32, true, true, FP8MLP_E4M3, FP8MLP_E5M2, tmA, tmB, tmB, a, c->sm_count, st));
+    }
+    // dX = dZq [W2q|W1q]^T
+    {
+        CUtensorMap tmA, tmB;
+        FP8MLP_TRY(make_tmap_u8(&tmA, c->dzq, 2 * f, T, 2 * f));
+        FP8MLP_TRY(make_tmap_u8(&tmB, c->w12q, 2 * f, d, 2 * f));
+        GemmArgs a = base_args(c, Ti, di, 2 * fi);
+        a.s0 = sc->dz; a.s1 = sc->w12;
+        a.out_bf16 = static_cast<uint16_t*>(dx);
+        FP8MLP_TRY(launch_gemm(EPI_BF16, false, false, FP8MLP_E5M2, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
+    }
+    // [dW2 | dW1] = Xq^T dZq
+    {
+        CUtensorMap tmA, tmB;
+        FP8MLP_TRY(make_tmap_u8(&tmA, c->xq, d, T, d));
+        FP8MLP_TRY(make_tmap_u8(&tmB, c->dzq, 2 * f, T, 2 * f));
+        GemmArgs a = base_args(c, di, 2 * fi, Ti);
+        a.s0 = sc->x; a.s1 = sc->dz;
+        a.out_f32_0 = dW2; a.out_f32_1 = dW1;
+        a.n_split = fi; a.ld_out = f;
+        FP8MLP_TRY(launch_gemm(EPI_F32, true, true, FP8MLP_E4M3, FP8MLP_E5M2, tmA, tmB, tmB, a, c->sm_count, st));
+    }
+    return FP8MLP_OK;
+}
+
+int fp8mlp_gemm_fp8(int64_t M, int64_t N, int64_t K, const uint8_t* A, int a_kmajor, int a_fmt, const uint8_t* B,
+                    int b_kmajor, int b_fmt, const float* scale_a, const float* scale_b, float* out, void* stream) {
+    if (A == nullptr || B == nullptr || out == nullptr) return FP8MLP_ERR_ARG;
+    if ((a_fmt != FP8MLP_E4M3 && a_fmt != FP8MLP_E5M2) || (b_fmt != FP8MLP_E4M3 && b_fmt != FP8MLP_E5M2)) return FP8MLP_ERR_ARG;
+    if (M <= 0 || N <= 0 || K <= 0 || M % 16 || N % 16 || K % 16 || M > (1 << 24) || N > (1 << 24) || K > (1 << 24)) return FP8MLP_ERR_SHAPE;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(out)) return FP8MLP_ERR_ALIGN;
+    int dev = 0, sms = 0;
+    FP8MLP_CUDA_CHECK(cudaGetDevice(&dev));
+    FP8MLP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CUtensorMap tmA, tmB;
+    if (a_kmajor) FP8MLP_TRY(make_tmap_u8(&tmA, A, K, M, K)); else FP8MLP_TRY(make_tmap_u8(&tmA, A, M, K, M));
+    if (b_kmajor) FP8MLP_TRY(make_tmap_u8(&tmB, B, K, N, K)); else FP8MLP_TRY(make_tmap_u8(&tmB, B, N, K, N));
+    GemmArgs a = base_args(nullptr, static_cast<int>(M), static_cast<int>(N), static_cast<int>(K));
+    a.s0 = scale_a; a.s1 = scale_b;
+    a.out_f32_0 = out; a.out_f32_1 = out;
+    return launch_gemm(EPI_F32, !a_kmajor, !b_kmajor, a_fmt, b_fmt, tmA, tmB, tmB, a, sms, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

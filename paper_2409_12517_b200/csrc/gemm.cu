@@ -1,0 +1,496 @@
+// tcgen05 FP8 GEMM kernel and its fused epilogues (see gemm.cuh for the design).
+#include "gemm.cuh"
+
+#include <mutex>
+
+namespace fp8mlp {
+
+namespace {
+
+// ---------------------------------------------------------------- shared memory plan
+struct __align__(8) SmemTail {
+    uint64_t full[kStages];      // TMA -> MMA: stage filled
+    uint64_t empty[kStages];     // MMA -> TMA: stage drained
+    uint64_t tmem_full[2];       // MMA -> epilogue: accumulator complete
+    uint64_t tmem_empty[2];      // epilogue -> MMA: accumulator drained
+    uint32_t tmem_base;
+    int abort;
+    float s_tile[2][kBlockN];    // per-channel scales of the current tile(s)
+    unsigned int amax_tile[128]; // per-channel maxima of the current tile (forward)
+};
+constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + size_t(kStages) * kStageBytes + sizeof(SmemTail);
+
+// ---------------------------------------------------------------- descriptors
+// Shared-memory matrix descriptor, 128-byte swizzle.  Bits: [0,14) address>>4, [16,30) leading
+// byte offset>>4, [32,46) stride byte offset>>4, [46,48) version 1, [61,64) layout 2 = SW128.
+//   K-major : rows 128 bytes apart, 8-row atoms 1024 bytes apart (stride offset); leading unused.
+//   MN-major: each K row holds 128 contiguous M/N bytes; 8-K-row atoms 1024 bytes apart (stride
+//             offset); the next 128 M/N bytes start one box (16 KiB) later (leading offset).
+template <bool MN_MAJOR>
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    constexpr uint64_t lbo = MN_MAJOR ? (kBoxBytes >> 4) : 1;
+    constexpr uint64_t sbo = 1024 >> 4;
+    return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+// Byte step of the descriptor start address per 32-element slice of K.
+template <bool MN_MAJOR>
+__device__ __forceinline__ uint32_t k_step_bytes() { return MN_MAJOR ? 32u * 128u : 32u; }
+
+__device__ __forceinline__ void tile_coords(const GemmArgs& p, int tile, int& m_tile, int& n_tile) {
+    // bands of group_m m-tiles; inside a band consecutive tiles walk down m first, so the CTAs
+    // running at the same time share a few A row-blocks and a few B column-blocks in L2
+    const int per_band = p.group_m * p.num_n_tiles;
+    const int band = tile / per_band;
+    const int first_m = band * p.group_m;
+    const int rows = min(p.num_m_tiles - first_m, p.group_m);
+    const int in_band = tile - band * per_band;
+    m_tile = first_m + in_band % rows;
+    n_tile = in_band / rows;
+}
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+// all epilogue threads agree on one predicate (and of all)
+__device__ __forceinline__ bool epi_all(bool v) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t"
+        "}\n"
+        : "=r"(r) : "r"(static_cast<uint32_t>(v)), "n"(kEpiThreads) : "memory");
+    return r != 0;
+}
+
+__device__ __forceinline__ float inv_or_one(const float* s) { return s ? __fdiv_rn(1.0f, *s) : 1.0f; }
+
+// ---------------------------------------------------------------- epilogues (one thread = one row)
+__device__ __forceinline__ void epilogue_f32(const GemmArgs& p, uint32_t taddr, int m, int n0, float dq) {
+    const bool row_ok = m < p.M;
+#pragma unroll 1
+    for (int j = 0; j < kBlockN / 32; ++j) {
+        const int c0 = n0 + 32 * j;
+        if (c0 >= p.N) break;
+        uint32_t r[32];
+        tmem_ld32(taddr + 32 * j, r);
+        tmem_ld_wait();
+        if (!row_ok) continue;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int col = c0 + 4 * q;
+            if (col < p.N) {
+                float* dst = col < p.n_split ? p.out_f32_0 + static_cast<int64_t>(m) * p.ld_out + col
+                                             : p.out_f32_1 + static_cast<int64_t>(m) * p.ld_out + (col - p.n_split);
+                st_global_v4(dst, __float_as_uint(__fmul_rn(__uint_as_float(r[4 * q + 0]), dq)),
+                             __float_as_uint(__fmul_rn(__uint_as_float(r[4 * q + 1]), dq)),
+                             __float_as_uint(__fmul_rn(__uint_as_float(r[4 * q + 2]), dq)),
+                             __float_as_uint(__fmul_rn(__uint_as_float(r[4 * q + 3]), dq)));
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void epilogue_bf16(const GemmArgs& p, uint32_t taddr, int m, int n0, float dq) {
+    const bool row_ok = m < p.M;
+#pragma unroll 1
+    for (int j = 0; j < kBlockN / 32; ++j) {
+        const int c0 = n0 + 32 * j;
+        if (c0 >= p.N) break;
+        uint32_t r[32];
+        tmem_ld32(taddr + 32 * j, r);
+        tmem_ld_wait();
+        if (!row_ok) continue;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int col = c0 + 8 * q;
+            if (col < p.N) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    w[e] = cvt_bf16x2(__fmul_rn(__uint_as_float(r[8 * q + 2 * e]), dq),
+                                      __fmul_rn(__uint_as_float(r[8 * q + 2 * e + 1]), dq));
+                st_global_v4(p.out_bf16 + static_cast<int64_t>(m) * p.ld_out + col, w[0], w[1], w[2], w[3]);
+            }
+        }
+    }
+}
+
+// Forward: accumulator columns [0,128) are G = x W2 (gate), [128,256) are U = x W1 (linear) of the
+// same 128 channels.  H = U * G * sigma(G); per-channel max |H|; Hq = Q_e4m3(H * s_i); bf16 G, U kept
+// for backward.  H itself never leaves the SM.
+__device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail* tail, uint32_t taddr, int lane,
+                                                    int m, int n0, float dq) {
+    const bool row_ok = m < p.M;
+    const int f = p.N;
+#pragma unroll 1
+    for (int j = 0; j < 4; ++j) {
+        const int c0 = n0 + 32 * j;
+        if (c0 >= f) break;
+        uint32_t g_raw[32], u_raw[32];
+        tmem_ld32(taddr + 32 * j, g_raw);
+        tmem_ld32(taddr + 128 + 32 * j, u_raw);
+        tmem_ld_wait();
+        float hs[32];
+        float colmax = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const float g = __fmul_rn(__uint_as_float(g_raw[e]), dq);
+            const float u = __fmul_rn(__uint_as_float(u_raw[e]), dq);
+            const float sw = __fmul_rn(g, sigmoid_f32(g));
+            const float h = __fmul_rn(u, sw);
+            const float cm = warp_max_nonneg(fabsf(h));       // max over this warp's 32 rows
+            if (lane == e) colmax = cm;
+            hs[e] = __fmul_rn(h, tail->s_tile[0][32 * j + e]);
+            g_raw[e] = __float_as_uint(g);
+            u_raw[e] = __float_as_uint(u);
+        }
+        atomicMax(&tail->amax_tile[32 * j + lane], __float_as_uint(colmax));
+        if (!p.store || !row_ok) continue;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int col = c0 + 16 * q;
+            if (col < f) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    w[e] = cvt_fp8x4<FP8MLP_E4M3>(hs[16 * q + 4 * e], hs[16 * q + 4 * e + 1], hs[16 * q + 4 * e + 2],
+                                                 hs[16 * q + 4 * e + 3]);
+                st_global_v4(p.hq + static_cast<int64_t>(m) * f + col, w[0], w[1], w[2], w[3]);
+            }
+        }
+        if (p.gu != nullptr) {
+            uint16_t* grow = p.gu + static_cast<int64_t>(m) * 2 * f;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int col = c0 + 8 * q;
+                if (col < f) {
+                    uint32_t wg[4], wu[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        wg[e] = cvt_bf16x2(__uint_as_float(g_raw[8 * q + 2 * e]), __uint_as_float(g_raw[8 * q + 2 * e + 1]));
+                        wu[e] = cvt_bf16x2(__uint_as_float(u_raw[8 * q + 2 * e]), __uint_as_float(u_raw[8 * q + 2 * e + 1]));
+                    }
+                    st_global_v4(grow + col, wg[0], wg[1], wg[2], wg[3]);
+                    st_global_v4(grow + f + col, wu[0], wu[1], wu[2], wu[3]);
+                }
+            }
+        }
+    }
+}
+
+// Backward: accumulator = dY W3'^T for 256 channels.  dH = acc * dq (* s_i with Smooth-SwiGLU);
+// dU = dH * G sigma(G); dG = dH * U * sigma(G) (1 + G (1 - sigma(G))); max of |dG|, |dU|;
+// dZq = Q_e5m2([dG | dU] * sdz).
+__device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const float* s_tile, uint32_t taddr, int m,
+                                                     int n0, float dq, float sdz) {
+    const bool row_ok = m < p.M;
+    const int f = p.N;
+    float local_max = 0.0f;
+#pragma unroll 1
+    for (int j = 0; j < kBlockN / 32; ++j) {
+        const int c0 = n0 + 32 * j;
+        if (c0 >= f) break;
+        uint32_t acc[32];
+        tmem_ld32(taddr + 32 * j, acc);
+        uint4 gq[4], uq[4];
+        const uint16_t* grow = p.gu + static_cast<int64_t>(m) * 2 * f + c0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const bool ok = row_ok && (c0 + 8 * q) < f;
+            gq[q] = ok ? ld_global_nc_v4(grow + 8 * q) : make_uint4(0, 0, 0, 0);
+            uq[q] = ok ? ld_global_nc_v4(grow + f + 8 * q) : make_uint4(0, 0, 0, 0);
+        }
+        tmem_ld_wait();
+        float dg[32], du[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const uint32_t gw = reinterpret_cast<const uint32_t*>(gq)[e >> 1];
+            const uint32_t uw = reinterpret_cast<const uint32_t*>(uq)[e >> 1];
+            const float g = (e & 1) ? bf16_hi(gw) : bf16_lo(gw);
+            const float u = (e & 1) ? bf16_hi(uw) : bf16_lo(uw);
+            float dh = __fmul_rn(__uint_as_float(acc[e]), dq);
+            if (p.smooth) dh = __fmul_rn(dh, s_tile[32 * j + e]);
+            const float sig = sigmoid_f32(g);
+            const float sw = __fmul_rn(g, sig);
+            du[e] = __fmul_rn(dh, sw);
+            const float t1 = __fadd_rn(1.0f, __fmul_rn(g, __fsub_rn(1.0f, sig)));
+            const float dsw = __fmul_rn(sig, t1);
+            dg[e] = __fmul_rn(__fmul_rn(dh, u), dsw);
+            local_max = fmaxf(local_max, fmaxf(fabsf(dg[e]), fabsf(du[e])));
+        }
+        if (!p.store || !row_ok) continue;
+        uint8_t* zrow = p.dzq + static_cast<int64_t>(m) * 2 * f + c0;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            if (c0 + 16 * q < f) {
+                uint32_t wg[4], wu[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int b = 16 * q + 4 * e;
+                    wg[e] = cvt_fp8x4<FP8MLP_E5M2>(__fmul_rn(dg[b], sdz), __fmul_rn(dg[b + 1], sdz),
+                                                  __fmul_rn(dg[b + 2], sdz), __fmul_rn(dg[b + 3], sdz));
+                    wu[e] = cvt_fp8x4<FP8MLP_E5M2>(__fmul_rn(du[b], sdz), __fmul_rn(du[b + 1], sdz),
+                                                  __fmul_rn(du[b + 2], sdz), __fmul_rn(du[b + 3], sdz));
+                }
+                st_global_v4(zrow + 16 * q, wg[0], wg[1], wg[2], wg[3]);
+                st_global_v4(zrow + f + 16 * q, wu[0], wu[1], wu[2], wu[3]);
+            }
+        }
+    }
+    return local_max;
+}
+
+// ---------------------------------------------------------------- the kernel
+template <int EPI, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+            const __grid_constant__ CUtensorMap tmB1, const GemmArgs p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;         // swizzle atoms need 1024-byte alignment
+    uint8_t* tiles_ptr = smem_raw + (tiles_addr - raw_addr);
+    SmemTail* tail = reinterpret_cast<SmemTail*>(tiles_ptr + size_t(kStages) * kStageBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_tiles = p.num_m_tiles * p.num_n_tiles;
+    volatile int* abort_flag = &tail->abort;
+
+    if (threadIdx.x == 0) {
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB0);
+        tma_prefetch_desc(&tmB1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&tail->full[s]), 1);
+            mbar_init(smem_u32(&tail->empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&tail->tmem_full[b]), 1);
+            mbar_init(smem_u32(&tail->tmem_empty[b]), kEpiThreads / 32);
+        }
+        tail->abort = 0;
+        mbar_init_fence();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tail->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                int m_tile, n_tile;
+                tile_coords(p, tile, m_tile, n_tile);
+                const int m0 = m_tile * kBlockM;
+                const int nb0 = n_tile * p.n_tile_cols;
+                const int nb1 = nb0 + p.b1_offset;
+                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                    if (!mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    const uint32_t bar = smem_u32(&tail->full[stage]);
+                    const uint32_t dst = tiles_addr + stage * kStageBytes;
+                    const int k0 = kb * kBlockK;
+                    mbar_expect_tx(bar, kStageBytes);
+                    if (A_MN) tma_load_2d(dst, &tmA, bar, m0, k0); else tma_load_2d(dst, &tmA, bar, k0, m0);
+                    if (B_MN) {
+                        tma_load_2d(dst + kBoxBytes, &tmB0, bar, nb0, k0);
+                        tma_load_2d(dst + 2 * kBoxBytes, &tmB1, bar, nb1, k0);
+                    } else {
+                        tma_load_2d(dst + kBoxBytes, &tmB0, bar, k0, nb0);
+                        tma_load_2d(dst + 2 * kBoxBytes, &tmB1, bar, k0, nb1);
+                    }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+                const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
+                if (!mbar_wait(smem_u32(&tail->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, p.status)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kBlockN;
+                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                    if (!mbar_wait(smem_u32(&tail->full[stage]), phase, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = tiles_addr + stage * kStageBytes;
+                    const uint32_t b_addr = a_addr + kBoxBytes;
+#pragma unroll
+                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                        const uint64_t da = smem_desc<A_MN>(a_addr + k * k_step_bytes<A_MN>());
+                        const uint64_t db = smem_desc<B_MN>(b_addr + k * k_step_bytes<B_MN>());
+                        umma_f8(d_tmem, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&tail->empty[stage]));      // frees the stage once these MMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(smem_u32(&tail->tmem_full[acc]));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int quad = warp & 3;                     // TMEM lanes [32*quad, 32*quad+32) belong to this warp
+        const int row = quad * 32 + lane;
+        const float dq0 = __fmul_rn(inv_or_one(p.s0), inv_or_one(p.s1));
+        float sdz = 1.0f;
+        if constexpr (EPI == EPI_SWIGLU_BWD) sdz = *p.sdz;
+        float run_max = 0.0f;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+            int m_tile, n_tile;
+            tile_coords(p, tile, m_tile, n_tile);
+            const int m = m_tile * kBlockM + row;
+            const int n0 = n_tile * p.n_tile_cols;
+            const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
+            if constexpr (EPI == EPI_SWIGLU_FWD) {
+                tail->s_tile[0][row] = (n0 + row) < p.N ? p.s_h[n0 + row] : 1.0f;
+                tail->amax_tile[row] = 0u;
+            }
+            if constexpr (EPI == EPI_SWIGLU_BWD) {
+                tail->s_tile[acc][row] = (n0 + row) < p.N ? p.s_h[n0 + row] : 1.0f;
+                tail->s_tile[acc][row + 128] = (n0 + row + 128) < p.N ? p.s_h[n0 + row + 128] : 1.0f;
+            }
+            const bool got = mbar_wait(smem_u32(&tail->tmem_full[acc]), acc_phase, abort_flag, p.status);
+            if (!epi_all(got)) break;                  // also orders the s_tile / amax_tile writes above
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + acc * kBlockN + (static_cast<uint32_t>(quad * 32) << 16);
+            if constexpr (EPI == EPI_F32) {
+                float dq = dq0;
+                if (p.row_s != nullptr)
+                    dq = __fmul_rn(inv_or_one(p.s0), m < p.M ? __fdiv_rn(1.0f, p.row_s[m]) : 1.0f);
+                epilogue_f32(p, taddr, m, n0, dq);
+            } else if constexpr (EPI == EPI_BF16) {
+                epilogue_bf16(p, taddr, m, n0, dq0);
+            } else if constexpr (EPI == EPI_SWIGLU_FWD) {
+                epilogue_swiglu_fwd(p, tail, taddr, lane, m, n0, dq0);
+            } else {
+                run_max = fmaxf(run_max, epilogue_swiglu_bwd(p, tail->s_tile[acc], taddr, m, n0, dq0, sdz));
+            }
+            // accumulator drained: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tail->tmem_empty[acc]));
+            if constexpr (EPI == EPI_SWIGLU_FWD) {
+                epi_bar_sync();                        // all four row quadrants have merged into amax_tile
+                const unsigned int v = tail->amax_tile[row];
+                if ((n0 + row) < p.N && v != 0u) atomicMax(p.amax_h + n0 + row, v);
+                // each thread resets only its own amax_tile / s_tile entry for the next tile, and the
+                // others touch them again only after the next tile's barrier: no second barrier needed
+            }
+        }
+        if constexpr (EPI == EPI_SWIGLU_BWD) {
+            run_max = warp_max_nonneg(run_max);
+            if (lane == 0 && run_max > 0.0f) atomicMax(p.amax_dz, __float_as_uint(run_max));
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies that are still in flight time to land before shared memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres);
+        if (e == cudaSuccess && qres == cudaDriverEntryPointSuccess) fn = reinterpret_cast<EncodeTiledFn>(sym);
+        else set_cuda_error("cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)", e);
+    });
+    return fn;
+}
+
+template <int EPI, bool A_MN, bool B_MN>
+int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorMap& tmB1, const GemmArgs& args,
+                int grid, cudaStream_t st) {
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(kSmemBytes));
+    });
+    FP8MLP_CUDA_CHECK(attr_err);
+    gemm_kernel<EPI, A_MN, B_MN><<<grid, kGemmThreads, kSmemBytes, st>>>(tmA, tmB0, tmB1, args);
+    FP8MLP_LAUNCH_CHECK();
+    return FP8MLP_OK;
+}
+
+}  // namespace
+
+size_t gemm_smem_bytes() { return kSmemBytes; }
+
+int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return FP8MLP_ERR_CUDA;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {row_stride};
+    const cuuint32_t box[2] = {128, 128};
+    const cuuint32_t elem[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_cuda_error_str("cuTensorMapEncodeTiled", "driver rejected the tensor map");
+        return FP8MLP_ERR_CUDA;
+    }
+    return FP8MLP_OK;
+}
+
+int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUtensorMap& tmA, const CUtensorMap& tmB0,
+                const CUtensorMap& tmB1, GemmArgs args, int sm_count, cudaStream_t st) {
+    args.num_m_tiles = (args.M + kBlockM - 1) / kBlockM;
+    args.num_n_tiles = (args.N + args.n_tile_cols - 1) / args.n_tile_cols;
+    args.num_k_blocks = (args.K + kBlockK - 1) / kBlockK;
+    if (args.group_m <= 0) args.group_m = 16;
+    // instruction descriptor: [4,6) D = fp32; [7,10) A format; [10,13) B format (0 = E4M3, 1 = E5M2);
+    // bit 15 / 16: A / B is MN-major; [17,23) N >> 3; [24,29) M >> 4
+    args.idesc = (1u << 4) | (static_cast<uint32_t>(a_fmt) << 7) | (static_cast<uint32_t>(b_fmt) << 10) |
+                 (static_cast<uint32_t>(a_mn) << 15) | (static_cast<uint32_t>(b_mn) << 16) |
+                 (static_cast<uint32_t>(kBlockN >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+    const int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
+    if (tiles == 0 || args.num_k_blocks == 0) return FP8MLP_OK;
+    const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);
+
+#define FP8MLP_DISPATCH(E, AM, BM) \
+    if (epi == E && a_mn == AM && b_mn == BM) return launch_inst<E, AM, BM>(tmA, tmB0, tmB1, args, grid, st);
+    FP8MLP_DISPATCH(EPI_F32, false, false)
+    FP8MLP_DISPATCH(EPI_F32, false, true)
+    FP8MLP_DISPATCH(EPI_F32, true, false)
+    FP8MLP_DISPATCH(EPI_F32, true, true)
+    FP8MLP_DISPATCH(EPI_BF16, false, false)
+    FP8MLP_DISPATCH(EPI_BF16, false, true)
+    FP8MLP_DISPATCH(EPI_SWIGLU_FWD, false, true)
+    FP8MLP_DISPATCH(EPI_SWIGLU_BWD, false, false)
+#undef FP8MLP_DISPATCH
+    return FP8MLP_ERR_ARG;
+}
+
+}  // namespace fp8mlp

@@ -1,0 +1,79 @@
+// FP8 GEMM for sm_100a: persistent, warp-specialised, tcgen05.mma kind::f8f6f4 with fp32
+// accumulators in tensor memory, operands streamed by TMA through a multi-stage shared-memory
+// ring, and the block's element-wise steps fused into the epilogue that drains tensor memory.
+//
+//   D[m, n] = sum_k A(m, k) * B(n, k)
+//
+// Either operand may be stored with K contiguous ("K-major", [rows, K]) or with its M/N index
+// contiguous ("MN-major", [K, rows]); both are fetched as 128-byte x 128-row TMA boxes with the
+// 128-byte swizzle and only the shared-memory matrix descriptors differ.  That lets the forward,
+// dgrad and wgrad GEMMs of the block all read the same FP8 buffers without transposed copies.
+//
+// CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the MMAs,
+// warps 2-5 are the epilogue (one TMEM lane quadrant each).  Two 256-column accumulators
+// alternate, so the epilogue of one tile overlaps the main loop of the next.
+// Every wait is bounded: on expiry the CTA raises a status word and drains.
+#pragma once
+
+#include "common.cuh"
+
+namespace fp8mlp {
+
+enum : int { EPI_F32 = 0, EPI_BF16 = 1, EPI_SWIGLU_FWD = 2, EPI_SWIGLU_BWD = 3 };
+
+constexpr int kBlockM = 128;          // rows of D per tile (TMEM lanes)
+constexpr int kBlockN = 256;          // accumulator columns per tile
+constexpr int kBlockK = 128;          // contraction elements (= bytes) per pipeline stage
+constexpr int kUmmaK = 32;            // contraction elements per tcgen05.mma (32 bytes)
+constexpr int kStages = 4;
+constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 bytes x 128 rows
+constexpr int kStageBytes = 3 * kBoxBytes;   // A box + two B boxes
+constexpr int kGemmThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr int kEpiThreads = 128;
+
+struct GemmArgs {
+    int M, N, K;            // N: extent of the n coordinate space (output columns; d_ff channels for the SwiGLU epilogues)
+    int num_m_tiles, num_n_tiles, num_k_blocks;
+    int n_tile_cols;        // n coordinates per tile: 256, or 128 when the two B boxes are gate and linear halves
+    int b1_offset;          // n offset of the second B box: 128, or 0 in the gate/linear case
+    int group_m;            // m-tiles per rasterisation band
+    uint32_t idesc;
+    int* status;
+
+    // dequantisation: dq = (1 / *s0) * (1 / *s1); a null pointer stands for 1
+    const float* s0;
+    const float* s1;
+    // EPI_F32: out = acc * dq; with row_s, dq = (1 / *s0) * (1 / row_s[m]).  Columns < n_split go to
+    // out_f32_0[m*ld_out + n], the others to out_f32_1[m*ld_out + n - n_split].
+    const float* row_s;
+    float* out_f32_0;
+    float* out_f32_1;
+    int n_split;
+    int64_t ld_out;
+    // EPI_BF16: out_bf16[m*ld_out + n] = bf16(acc * dq)
+    uint16_t* out_bf16;
+    // SwiGLU epilogues (f = N)
+    const float* s_h;       // [f] per-channel scale of H
+    int smooth;             // backward: multiply dH by s_h (Smooth-SwiGLU) or not (per-tensor scale)
+    int store;              // 0: calibration pass, only the maxima are produced
+    uint8_t* hq;            // fwd: E4M3 [M, f]
+    uint16_t* gu;           // fwd: out (nullable), bwd: in; bf16 [M, 2f] = G | U
+    unsigned int* amax_h;   // fwd: [f] bit patterns of max |H|, raised atomically
+    const float* sdz;       // bwd: scale of dZ
+    uint8_t* dzq;           // bwd: E5M2 [M, 2f] = dG | dU
+    unsigned int* amax_dz;  // bwd: bit pattern of max(|dG|, |dU|), raised atomically
+};
+
+size_t gemm_smem_bytes();
+
+// Encodes the 2-D tiled tensor map of an 8-bit matrix whose rows are `inner` bytes long and
+// `row_stride` bytes apart: box = 128 bytes x 128 rows, 128-byte swizzle, zero fill out of bounds.
+int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride);
+
+// Launches one GEMM.  a_mn / b_mn: the operand is MN-major.  The tensor maps describe A, and the
+// two 128-wide halves of the B tile (the same map twice unless they come from different matrices).
+int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUtensorMap& tmA,
+                const CUtensorMap& tmB0, const CUtensorMap& tmB1, GemmArgs args, int sm_count, cudaStream_t st);
+
+}  // namespace fp8mlp

@@ -1,0 +1,39 @@
+"""Shared helpers of the parity tests (no method arithmetic: comparisons and marshalling only)."""
+import numpy as np
+import torch
+
+
+def to_dev_bf16(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16).copy()).cuda().view(torch.bfloat16)
+
+
+def bf16_dev_to_bits(t: torch.Tensor) -> np.ndarray:
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def to_dev(a: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def code_rank(codes: np.ndarray) -> np.ndarray:
+    """FP8 codes (sign-magnitude) -> integers that order like the values they encode."""
+    c = codes.astype(np.int32)
+    mag = c & 0x7F
+    return np.where(c & 0x80, -mag, mag)
+
+
+def code_mismatch(got: np.ndarray, ref: np.ndarray):
+    """(fraction of differing codes, largest distance in code steps)."""
+    diff = np.abs(code_rank(got) - code_rank(ref))
+    return float(np.count_nonzero(diff)) / max(diff.size, 1), int(diff.max()) if diff.size else 0
+
+
+def nmax_err(got: np.ndarray, ref: np.ndarray) -> float:
+    """max |got - ref| / max |ref|."""
+    ref = ref.astype(np.float64)
+    denom = np.abs(ref).max()
+    return float(np.abs(got.astype(np.float64) - ref).max() / (denom if denom > 0 else 1.0))
+
+
+def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)

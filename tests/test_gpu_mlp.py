@@ -1,0 +1,176 @@
+"""Parity of fp8mlp_forward / fp8mlp_backward with the CPU oracle, element by element.
+
+Bars (from the benchmark definition): quantised inputs and amax bit-exact; SwiGLU codes at most
+1 code step apart on at most 0.1 % of elements (fp32 accumulation order and the exponential
+differ); Y, dX, dW within 2e-3 of the oracle's max |value|.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import bf16_dev_to_bits, bf16_bits_to_f32, code_mismatch, nmax_err, to_dev, to_dev_bf16
+from paper_2409_12517_b200 import binding as B
+from paper_2409_12517_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+CODE_FRAC = 1e-3
+OUT_TOL = 2e-3
+AMAX_RTOL = 1e-5
+
+
+class Run:
+    """One forward(+backward) through the C ABI with everything the oracle can be compared on."""
+
+    def __init__(self, w, flags, mode, given=None, backward=True):
+        T, d, f = w.T, w.d, w.f
+        self.w = w
+        self.smooth = bool(flags & B.SMOOTH)
+        self.ctx = B.fp8mlp_create(max(T, 1), d, f, flags)
+        self.sc, self.am = B.new_scales(f), B.new_amax(f)
+        if given is not None:
+            for k, v in given.items():
+                self.sc[k].copy_(to_dev(np.atleast_1d(np.asarray(v, np.float32))))
+        x = to_dev_bf16(w.x)
+        W1, W2, W3 = to_dev(w.W1), to_dev(w.W2), to_dev(w.W3)
+        y = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        B.fp8mlp_forward(self.ctx, T, x, W1, W2, W3, mode, self.sc, self.am, y)
+        self.Y_bits = bf16_dev_to_bits(y)
+        ws = lambda which, shape, dt=torch.uint8: B.workspace_tensor(self.ctx, which, shape, dt).cpu().numpy()
+        self.Xq, self.W12q = ws(B.WS_XQ, (T, d)), ws(B.WS_W12Q, (d, 2 * f))
+        self.W3q, self.Hq = ws(B.WS_W3Q, (f, d)), ws(B.WS_HQ, (T, f))
+        if flags & B.SAVE_FOR_BWD:
+            self.GU = B.workspace_tensor(self.ctx, B.WS_GU, (T, 2 * f), torch.int16).cpu().numpy().view(np.uint16)
+        if backward:
+            dy = to_dev_bf16(w.dY)
+            dx = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+            self.dW1 = torch.full((d, f), float("nan"), device="cuda")
+            self.dW2 = torch.full((d, f), float("nan"), device="cuda")
+            self.dW3 = torch.full((f, d), float("nan"), device="cuda")
+            B.fp8mlp_backward(self.ctx, T, dy, mode, self.sc, self.am, dx, self.dW1, self.dW2, self.dW3)
+            self.dX_bits = bf16_dev_to_bits(dx)
+            self.dYq, self.dZq = ws(B.WS_DYQ, (T, d)), ws(B.WS_DZQ, (T, 2 * f))
+        assert B.fp8mlp_status(self.ctx) == B.OK
+        self.scales = {k: v.cpu().numpy() for k, v in self.sc.items()}
+        self.amax = {k: v.cpu().numpy() for k, v in self.am.items()}
+
+    def close(self):
+        B.fp8mlp_destroy(self.ctx)
+
+
+def check_forward(r: Run, fw: dict, save=True):
+    f = r.w.f
+    assert r.scales["x"][0] == np.float32(fw["sx"]) and r.scales["w12"][0] == np.float32(fw["sw12"])
+    assert r.amax["x"][0] == np.float32(fw["amax_x"])
+    assert r.amax["w1"][0] == np.float32(fw["amax_w1"]) and r.amax["w2"][0] == np.float32(fw["amax_w2"])
+    assert np.array_equal(r.Xq, fw["Xq"]), "x codes differ"
+    assert np.array_equal(r.W12q, fw["W12q"]), "[W2|W1] codes differ"
+    assert np.allclose(r.amax["h"], fw["amax_h"], rtol=AMAX_RTOL, atol=0), "per-channel amax of H"
+    if r.smooth:
+        assert np.array_equal(r.scales["h"], fw["s_h"]), "per-channel scales s_i"
+    else:   # 448 / max amax_h inherits the last-bit difference of amax_h (accumulation order)
+        assert np.allclose(r.scales["h"], fw["s_h"], rtol=AMAX_RTOL, atol=0), "per-tensor scale of H"
+    assert r.amax["w3"][0] == np.float32(fw["amax_w3"]) and r.scales["w3"][0] == np.float32(fw["sw3"])
+    assert np.array_equal(r.W3q, fw["W3q"]), "W3' codes differ"
+    frac, worst = code_mismatch(r.Hq, fw["Hq"])
+    assert worst <= 1 and frac <= CODE_FRAC, f"Hq codes: {frac:.2e} differ, worst {worst} steps"
+    if save:
+        for name, got, ref in (("G", r.GU[:, :f], fw["G"]), ("U", r.GU[:, f:], fw["U"])):
+            e = nmax_err(bf16_bits_to_f32(got), bf16_bits_to_f32(ref))
+            assert e <= 2.0 ** -8, f"saved {name}: {e}"
+    e = nmax_err(bf16_bits_to_f32(r.Y_bits), fw["Y"])
+    assert e <= OUT_TOL, f"Y: {e}"
+
+
+def check_backward(r: Run, bw: dict):
+    assert r.amax["dy"][0] == np.float32(bw["amax_dy"]) and r.scales["dy"][0] == np.float32(bw["sdy"])
+    assert np.array_equal(r.dYq, bw["dYq"]), "dY codes differ"
+    assert np.isclose(r.amax["dz"][0], bw["amax_dz"], rtol=1e-3), "amax of dZ"
+    assert r.scales["dz"][0] == np.float32(bw["sdz"]), "scale of dZ"
+    frac, worst = code_mismatch(r.dZq, bw["dZq"])
+    assert worst <= 1 and frac <= CODE_FRAC, f"dZq codes: {frac:.2e} differ, worst {worst} steps"
+    for name, got, ref in (("dX", bf16_bits_to_f32(r.dX_bits), bw["dX"]), ("dW1", r.dW1.cpu().numpy(), bw["dW1"]),
+                           ("dW2", r.dW2.cpu().numpy(), bw["dW2"]), ("dW3", r.dW3.cpu().numpy(), bw["dW3"])):
+        assert np.all(np.isfinite(got)), f"{name} has unwritten or non-finite entries"
+        e = nmax_err(got, ref)
+        assert e <= OUT_TOL, f"{name}: {e}"
+
+
+def _oracle_flags(flags):
+    return oracle.FLAG_SMOOTH if flags & B.SMOOTH else 0
+
+
+@pytest.mark.parametrize("flags", [B.SMOOTH | B.SAVE_FOR_BWD, B.SAVE_FOR_BWD])
+def test_tiny_config_current_amax(flags):
+    """The tiny benchmark configuration (T=128, d=256, f=704: 5.5 channel tiles), scales from the
+    current amax, Smooth-SwiGLU on and off."""
+    w = wl.make_config("tiny")
+    fw = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=_oracle_flags(flags))
+    bw = oracle.backward(fw, w.dY)
+    r = Run(w, flags, B.SCALE_FROM_CURRENT_AMAX)
+    try:
+        check_forward(r, fw)
+        check_backward(r, bw)
+    finally:
+        r.close()
+
+
+@pytest.mark.parametrize("shape", [(200, 320, 272), (1, 16, 16), (130, 144, 528), (333, 512, 1040)])
+def test_ragged_shapes_given_scales(shape):
+    """Several tiles with ragged tails in every dimension, delayed-scaling mode: scales come from an
+    oracle run on other data (a previous step), so values also saturate and underflow."""
+    T, d, f = shape
+    w = wl.make("r", 11, T, d, f, w_std=0.05, channel_outlier_frac=0.01, token_outlier_frac=0.02)
+    prev = wl.make("p", 12, T, d, f, w_std=0.05)
+    pf = oracle.forward(prev.x, w.W1, w.W2, w.W3)
+    pb = oracle.backward(pf, prev.dY)
+    given = dict(x=pf["sx"], w12=pf["sw12"], w3=pf["sw3"], h=pf["s_h"], dy=pb["sdy"], dz=pb["sdz"])
+    fw = oracle.forward(w.x, w.W1, w.W2, w.W3, scale_mode=oracle.SCALE_GIVEN, sx=pf["sx"], sw12=pf["sw12"],
+                        s_h=pf["s_h"], sw3=pf["sw3"])
+    bw = oracle.backward(fw, w.dY, scale_mode=oracle.SCALE_GIVEN, sdy=pb["sdy"], sdz=pb["sdz"])
+    r = Run(w, B.SMOOTH | B.SAVE_FOR_BWD, B.SCALE_GIVEN, given=given)
+    try:
+        for k, v in given.items():                       # given scales are left alone
+            assert np.array_equal(r.scales[k], np.atleast_1d(np.asarray(v, np.float32)))
+        check_forward(r, fw)
+        check_backward(r, bw)
+    finally:
+        r.close()
+
+
+def test_forward_only_context_and_state_errors():
+    w = wl.make("s", 2, 64, 128, 256, w_std=0.05)
+    fw = oracle.forward(w.x, w.W1, w.W2, w.W3)
+    r = Run(w, B.SMOOTH, B.SCALE_FROM_CURRENT_AMAX, backward=False)
+    try:
+        check_forward(r, fw, save=False)
+        dx = torch.zeros((w.T, w.d), dtype=torch.bfloat16, device="cuda")
+        g = torch.zeros((w.d, w.f), device="cuda")
+        g3 = torch.zeros((w.f, w.d), device="cuda")
+        with pytest.raises(B.Fp8MlpError) as ei:
+            B.fp8mlp_backward(r.ctx, w.T, to_dev_bf16(w.dY), B.SCALE_GIVEN, r.sc, r.am, dx, g, g, g3)
+        assert ei.value.code == B.ERR_STATE
+        with pytest.raises(B.Fp8MlpError) as ei:
+            B.fp8mlp_forward(r.ctx, w.T + 1, to_dev_bf16(w.x), to_dev(w.W1), to_dev(w.W2), to_dev(w.W3),
+                             B.SCALE_GIVEN, r.sc, r.am, dx)
+        assert ei.value.code == B.ERR_SHAPE
+    finally:
+        r.close()
+
+
+def test_empty_batch():
+    w = wl.make("e", 2, 16, 64, 64, w_std=0.05)
+    ctx = B.fp8mlp_create(16, 64, 64, B.SMOOTH | B.SAVE_FOR_BWD)
+    try:
+        sc, am = B.new_scales(64), B.new_amax(64)
+        W1, W2, W3 = to_dev(w.W1), to_dev(w.W2), to_dev(w.W3)
+        B.fp8mlp_forward(ctx, 0, None, W1, W2, W3, B.SCALE_FROM_CURRENT_AMAX, sc, am, None)
+        g1, g2, g3 = (torch.full((64, 64), 7.0, device="cuda") for _ in range(3))
+        B.fp8mlp_backward(ctx, 0, None, B.SCALE_FROM_CURRENT_AMAX, sc, am, None, g1, g2, g3)
+        torch.cuda.synchronize()
+        assert float(g1.abs().max()) == 0 and float(g2.abs().max()) == 0 and float(g3.abs().max()) == 0
+        assert am["x"].item() == 0 and float(am["h"].max()) == 0
+        assert am["w1"].item() == oracle.amax(w.W1)
+    finally:
+        B.fp8mlp_destroy(ctx)
