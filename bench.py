@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark of the FP8 Smooth-SwiGLU MLP block (forward + backward) on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--workload 7b] [--impl reference]
+
+A step is one pass of the whole hot path over one synthetic batch: quantise x, W1/W2, W3' and
+dY, the gate/up GEMM with the Smooth-SwiGLU epilogue, the down projection, and the four backward
+GEMMs, in delayed-scaling mode (scales given, maxima emitted), as in steady-state training.
+Metric: TFLOP/s = 18*T*d*f / time.  One JSON line is printed by rank 0.
+
+N > 1 (launched by torch.distributed.run): the block has no exchange step on one GPU and the
+benchmark definition runs it on one GPU, so N ranks run N independent replicas (weak scaling);
+the only collective is the barrier / max-reduction of the timing.
+
+--impl reference times the CPU oracle (oracle/), as it stands, on a bounded sample of the
+same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "FP8 Smooth-SwiGLU MLP fwd+bwd TFLOP/s (7B shape); % of B200 dense FP8 peak"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+FP8_OVER_BF16 = 2.0          # nominal dense tensor-core ratio (4.5 vs 2.25 PFLOP/s)
+NOMINAL_FP8_TFLOPS = 4500.0
+# DRAM bytes per launch of the dominant kernel (gate/up GEMM + SwiGLU epilogue) measured by ncu
+# (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None until captured.
+NCU_TRAFFIC_BYTES = {"7b": None}
+
+
+def flops_step(T, d, f):
+    return 18.0 * T * d * f
+
+
+def load_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        return json.loads(p.read_text()), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ---------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.thread, self.gpu = [], None, None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 and len(r) >= 8] or [r for _, r in self.rows if len(r) >= 8]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        num = lambda s: float(s) if s.replace(".", "", 1).isdigit() else None
+        sm = sorted(v for v in (num(r[0]) for r in rows) if v is not None)
+        reasons = set()
+        for r in rows:
+            for name, col in (("hw_slowdown", 4), ("hw_thermal_slowdown", 5), ("sw_thermal_slowdown", 6), ("sw_power_cap", 7)):
+                if r[col].lower().startswith("active"):
+                    reasons.add(name)
+        power = [v for v in (num(r[2]) for r in rows) if v is not None]
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": num(rows[0][1]),
+                "power_w_max": max(power) if power else None, "samples": len(rows), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------- CPU oracle timing
+def time_oracle(w, T_s: int, f_s: int):
+    """One forward + backward of the oracle on the first T_s tokens and f_s channels; seconds."""
+    import oracle
+    x, dy = w.x[:T_s], w.dY[:T_s]
+    W1, W2, W3 = w.W1[:, :f_s], w.W2[:, :f_s], w.W3[:f_s, :]
+    t = time.perf_counter()
+    fw = oracle.forward(x, W1, W2, W3)
+    oracle.backward(fw, dy)
+    return time.perf_counter() - t
+
+
+def cpu_baseline(w, seconds_target: float = 20.0):
+    import oracle
+    cores = oracle.num_threads()
+    T_s = min(w.T, max(4, 2 * cores))
+    f_s = w.f
+    dt = time_oracle(w, T_s, f_s)
+    return {"value": flops_step(T_s, w.d, f_s) / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"fwd+bwd of the first {T_s} tokens, all {f_s} channels ({dt:.1f} s)"}
+
+
+def run_reference(args, rank: int):
+    """The CPU oracle as the reference arm: K timed steps, each a bounded sample of the workload."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2409_12517_b200 import workloads as wl
+    cfg = dict(wl.CONFIGS[args.workload])
+    cores = oracle.num_threads()
+    T_s = min(cfg["T"], max(4, 2 * cores))
+    w = wl.make_config(args.workload, T=T_s)            # same seed: the first T_s tokens of the workload
+    # size the channel sample so that the whole run stays within a couple of minutes
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    f_s = 256
+    t_probe = time_oracle(w, T_s, f_s)
+    f_s = int(min(w.f, max(256, 256 * int(budget / max(t_probe, 1e-3)))))
+    for _ in range(args.warmup):
+        time_oracle(w, T_s, f_s)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time_oracle(w, T_s, f_s)
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    value = flops_step(T_s, w.d, f_s) / dt / 1e12
+    sample = f"each step: fwd+bwd of the first {T_s} tokens and first {f_s} of {w.f} channels"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "fp8 (emulated on the CPU, fp32 accumulate)", "data": "synthetic",
+        "config": {"workload": args.workload, "T": cfg["T"], "d_model": w.d, "d_ff": w.f, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ---------------------------------------------------------------- the CUDA arm
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import numpy as np
+    import torch
+
+    from paper_2409_12517_b200 import binding as B
+    from paper_2409_12517_b200 import build as libbuild
+    from paper_2409_12517_b200 import workloads as wl
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    libbuild.build()
+    B.lib()
+
+    w = wl.make_config(args.workload)
+    T, d, f = w.T, w.d, w.f
+    dev_bf16 = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    x, dy = dev_bf16(w.x), dev_bf16(w.dY)
+    W1, W2, W3 = (torch.from_numpy(a).cuda() for a in (w.W1, w.W2, w.W3))
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    dW1, dW2, dW3 = torch.empty_like(W1), torch.empty_like(W2), torch.empty_like(W3)
+    ctx = B.fp8mlp_create(T, d, f, B.SMOOTH | B.SAVE_FOR_BWD)
+    sc, am = B.new_scales(f), B.new_amax(f)
+
+    def step(mode=B.SCALE_GIVEN):
+        B.fp8mlp_forward(ctx, T, x, W1, W2, W3, mode, sc, am, y)
+        B.fp8mlp_backward(ctx, T, dy, mode, sc, am, dx, dW1, dW2, dW3)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # the "previous iteration" that delayed scaling takes its scales from: one just-in-time step
+    step(B.SCALE_FROM_CURRENT_AMAX)
+    for _ in range(args.warmup):
+        step()
+    assert B.fp8mlp_status(ctx) == B.OK
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    B.fp8mlp_profile_enable(ctx, True)
+    B.fp8mlp_profile_read(ctx)
+    barrier()
+    n0 = B.fp8mlp_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    launches = B.fp8mlp_launch_count() - n0
+    ms_total = e0.elapsed_time(e1)
+    prof = B.fp8mlp_profile_read(ctx)
+    B.fp8mlp_profile_enable(ctx, False)
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    assert B.fp8mlp_status(ctx) == B.OK
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * flops_step(T, d, f) / (ms_step * 1e-3) / 1e12
+
+    # end to end: inputs start in pinned host memory, results end in host memory, every step
+    xh, dyh = x.cpu().pin_memory(), dy.cpu().pin_memory()
+    yh, dxh = torch.empty_like(xh).pin_memory(), torch.empty_like(xh).pin_memory()
+
+    def e2e_step():
+        x.copy_(xh, non_blocking=True)
+        B.fp8mlp_forward(ctx, T, x, W1, W2, W3, B.SCALE_GIVEN, sc, am, y)
+        yh.copy_(y, non_blocking=True)
+        dy.copy_(dyh, non_blocking=True)
+        B.fp8mlp_backward(ctx, T, dy, B.SCALE_GIVEN, sc, am, dx, dW1, dW2, dW3)
+        dxh.copy_(dx, non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 10))
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    B.fp8mlp_destroy(ctx)
+    if rank != 0:
+        return
+
+    peaks, peak_kind = load_peaks()
+    fp8_peak = FP8_OVER_BF16 * peaks["bf16_tflops_sustained"]       # kernels timed inside a long step
+    # per-phase table: GEMMs in TFLOP/s, quantise kernels in GB/s (algorithmic bytes)
+    tdf = float(T) * d * f
+    phase_flops = {"gemm1_swiglu": 4 * tdf, "gemm2_down": 2 * tdf, "dgrad2_swiglu_bwd": 2 * tdf, "wgrad3": 2 * tdf,
+                   "dgrad1": 4 * tdf, "wgrad12": 4 * tdf}
+    phase_bytes = {"quant_x": 3.0 * T * d, "quant_dy": 3.0 * T * d, "quant_w12": 5.0 * 2 * d * f, "quant_w3": 5.0 * d * f}
+    kernels = {}
+    for name, (ms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        avg = ms / cnt
+        entry = {"ms": round(avg, 4), "per_step": cnt / args.steps}
+        if name in phase_flops:
+            entry["tflops"] = round(phase_flops[name] / (avg * 1e-3) / 1e12, 1)
+            entry["frac_of_fp8_peak"] = round(entry["tflops"] / fp8_peak, 3)
+        if name in phase_bytes:
+            entry["gbs"] = round(phase_bytes[name] / (avg * 1e-3) / 1e9, 1)
+            entry["frac_of_hbm_peak"] = round(entry["gbs"] / peaks["hbm_gbs"], 3)
+        kernels[name] = entry
+    dom = "gemm1_swiglu"
+    achieved = kernels[dom]["tflops"]
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": fp8_peak, "unit": "TFLOP/s",
+                "frac": round(achieved / fp8_peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                "peak_source": f"of {peak_kind}: 2 x bf16_tflops_sustained ({peaks['bf16_tflops_sustained']}) "
+                               "- no FP8 GEMM peak is measured on this pool, the nominal FP8:bf16 ratio is applied",
+                "frac_of_nominal_fp8_4500": round(achieved / NOMINAL_FP8_TFLOPS, 4),
+                "step_frac_of_peak": round(value / world / fp8_peak, 4),
+                "quantize_hbm_frac": {k: v["frac_of_hbm_peak"] for k, v in kernels.items() if "gbs" in v},
+                "hbm_peak_gbs": peaks["hbm_gbs"]}
+    h2d = 2 * T * d * 2
+    d2h = 2 * T * d * 2
+    out = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "fp8 (E4M3 fwd / E5M2 grads, fp32 accumulate)", "data": "synthetic",
+        "config": {"workload": args.workload, "T": T, "d_model": d, "d_ff": f, "smooth_swiglu": True,
+                   "scale_mode": "given (delayed), maxima emitted every step", "replicas": world,
+                   "l2": "inputs per step (fp32 master weights 541 MB at the 7B shape) exceed the 126 MB L2"},
+        "clocks": clocks,
+        "e2e": {"value": round(world * flops_step(T, d, f) / (e2e_ms * 1e-3) / 1e12, 2), "unit": UNIT,
+                "ms_per_step": round(e2e_ms, 4), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "what": "x and dY copied from pinned host memory, Y and dX copied back, weights resident"},
+        "gpu_launches": launches,
+        "roofline": roofline,
+        "kernels": kernels,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(w)
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="7b")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -68,6 +68,21 @@ enum { /* fp8mlp_workspace: internal buffers, for inspection by tests */
     FP8MLP_WS_DZQ = 6   /* E5M2 [T,2f]  quantised [dG | dU]                            */
 };
 
+enum { /* phases of one step, for fp8mlp_profile_read (SMOOTH-mode kernel sequence) */
+    FP8MLP_PH_QUANT_X = 0,    /* x -> E4M3 (+ amax)                                   */
+    FP8MLP_PH_QUANT_W12 = 1,  /* W2, W1 -> E4M3 [W2|W1] (+ amax)                      */
+    FP8MLP_PH_QUANT_W3 = 2,   /* 1/s, diag(1/s) W3 -> E4M3 (+ amax)                   */
+    FP8MLP_PH_GEMM1 = 3,      /* gate/up GEMM + SwiGLU / Smooth-SwiGLU epilogue       */
+    FP8MLP_PH_GEMM2 = 4,      /* down projection                                      */
+    FP8MLP_PH_QUANT_DY = 5,   /* dY -> E5M2 (+ amax)                                  */
+    FP8MLP_PH_DGRAD2 = 6,     /* dY W3'^T + SwiGLU-backward epilogue                  */
+    FP8MLP_PH_WGRAD3 = 7,     /* dW3                                                  */
+    FP8MLP_PH_DGRAD1 = 8,     /* dX                                                   */
+    FP8MLP_PH_WGRAD12 = 9,    /* dW2 | dW1                                            */
+    FP8MLP_PH_MISC = 10,      /* amax resets, scale updates                           */
+    FP8MLP_PH_COUNT = 11
+};
+
 /* The paper's scaling state (Section 2: per-tensor scaling, delayed or just-in-time; Section 4.4:
  * per-channel s_i).  Every member is a device pointer to float(s), caller-owned; the library
  * keeps no history.  A scale multiplies the tensor before the cast: code = Q(v * scale).
@@ -91,6 +106,13 @@ FP8MLP_API const char* fp8mlp_last_cuda_error(void);
 FP8MLP_API int fp8mlp_status(fp8mlp_ctx* ctx, void* stream);
 /* Device pointer and size in bytes of one of the FP8MLP_WS_* buffers (sized for T_max). */
 FP8MLP_API int fp8mlp_workspace(fp8mlp_ctx* ctx, int which, void** ptr, int64_t* bytes);
+/* Per-phase device timing (no counterpart in the paper; measurement support).  While enabled,
+ * forward/backward record a CUDA event pair around every phase on the caller's stream.
+ * fp8mlp_profile_read waits for the recorded events, adds their elapsed times into ms[phase]
+ * (milliseconds) and the number of recorded brackets into count[phase] (both arrays of
+ * FP8MLP_PH_COUNT entries, overwritten), and forgets them. */
+FP8MLP_API int fp8mlp_profile_enable(fp8mlp_ctx* ctx, int on);
+FP8MLP_API int fp8mlp_profile_read(fp8mlp_ctx* ctx, double* ms, int64_t* count);
 /* Number of kernels this library has launched in this process so far (all contexts). */
 FP8MLP_API int64_t fp8mlp_launch_count(void);
 

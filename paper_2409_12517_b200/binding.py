@@ -25,8 +25,10 @@ WS_XQ, WS_W12Q, WS_W3Q, WS_HQ, WS_GU, WS_DYQ, WS_DZQ = range(7)
 EXPORTS = [
     "fp8mlp_create", "fp8mlp_destroy", "fp8mlp_strerror", "fp8mlp_last_cuda_error", "fp8mlp_status",
     "fp8mlp_workspace", "fp8mlp_launch_count", "fp8mlp_quantize", "fp8mlp_update_scales",
-    "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8",
+    "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8", "fp8mlp_profile_enable", "fp8mlp_profile_read",
 ]
+PHASES = ["quant_x", "quant_w12", "quant_w3", "gemm1_swiglu", "gemm2_down", "quant_dy", "dgrad2_swiglu_bwd",
+          "wgrad3", "dgrad1", "wgrad12", "misc"]
 
 
 class Fp8MlpError(RuntimeError):
@@ -73,6 +75,8 @@ def lib():
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.fp8mlp_gemm_fp8.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int,
                                       C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.fp8mlp_profile_enable.argtypes = [C.c_void_p, C.c_int]
+        L.fp8mlp_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         missing = [name for name in EXPORTS if not hasattr(L, name)]
         if missing:
             raise RuntimeError(f"{LIB_PATH} does not export {missing}")
@@ -131,6 +135,18 @@ def fp8mlp_workspace(ctx: int, which: int):
     p, n = C.c_void_p(), C.c_int64()
     _check(lib().fp8mlp_workspace(C.c_void_p(ctx), which, C.byref(p), C.byref(n)), "fp8mlp_workspace")
     return p.value, n.value
+
+
+def fp8mlp_profile_enable(ctx: int, on: bool) -> None:
+    _check(lib().fp8mlp_profile_enable(C.c_void_p(ctx), int(on)), "fp8mlp_profile_enable")
+
+
+def fp8mlp_profile_read(ctx: int) -> dict:
+    """{phase name: (milliseconds, brackets)} accumulated since the last read."""
+    n = len(PHASES)
+    ms, cnt = (C.c_double * n)(), (C.c_int64 * n)()
+    _check(lib().fp8mlp_profile_read(C.c_void_p(ctx), ms, cnt), "fp8mlp_profile_read")
+    return {PHASES[i]: (float(ms[i]), int(cnt[i])) for i in range(n)}
 
 
 def fp8mlp_quantize(src, fp8_fmt: int, scale_mode: int, scale, amax, row_mul, dst, ld_dst: int | None = None) -> None:

@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "gemm.cuh"
 #include "quantize.cuh"
@@ -44,9 +45,39 @@ struct fp8mlp_ctx {
     int* status;      // bounded-wait status word
     int64_t saved_T;  // tokens of the last forward that saved activations, -1 if none
     int64_t bytes[7];
+    // per-phase timing
+    bool profiling;
+    struct Bracket { int phase; cudaEvent_t e0, e1; };
+    std::vector<Bracket>* brackets;      // recorded, not yet read
+    std::vector<cudaEvent_t>* free_events;
 };
 
 namespace {
+
+// Records an event pair around a phase of forward/backward when profiling is on.
+struct PhaseTimer {
+    fp8mlp_ctx* c;
+    cudaStream_t st;
+    fp8mlp_ctx::Bracket b;
+    bool on;
+    static cudaEvent_t take(fp8mlp_ctx* c) {
+        if (!c->free_events->empty()) { cudaEvent_t e = c->free_events->back(); c->free_events->pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+    PhaseTimer(fp8mlp_ctx* ctx, int phase, cudaStream_t s) : c(ctx), st(s), on(ctx->profiling) {
+        if (!on) return;
+        b.phase = phase; b.e0 = take(c); b.e1 = take(c);
+        if (b.e0 == nullptr || b.e1 == nullptr) { on = false; return; }
+        cudaEventRecord(b.e0, st);
+    }
+    ~PhaseTimer() {
+        if (!on) return;
+        cudaEventRecord(b.e1, st);
+        c->brackets->push_back(b);
+    }
+};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -88,6 +119,22 @@ GemmArgs base_args(fp8mlp_ctx* c, int M, int N, int K) {
     a.ld_out = N;
     a.store = 1;
     return a;
+}
+
+// [W2 | W1] -> E4M3 codes in the [d, 2f] layout (gate columns first), one scale for both halves
+int quantize_w12(fp8mlp_ctx* c, const float* W1, const float* W2, int mode, float* scale, float* a_w1, float* a_w2,
+                 cudaStream_t st) {
+    const int64_t d = c->d, f = c->f;
+    const int sms = c->sm_count;
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
+        FP8MLP_TRY(run_quantize_pass(false, true, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, nullptr, nullptr, 0, a_w1, sms, st));
+        FP8MLP_TRY(run_quantize_pass(false, true, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, nullptr, nullptr, 0, a_w2, sms, st));
+        FP8MLP_TRY(run_scale_from_amax(FP8MLP_E4M3, a_w1, a_w2, scale, st));
+        FP8MLP_TRY(run_quantize_pass(true, false, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, scale, c->w12q, 2 * f, nullptr, sms, st));
+        return run_quantize_pass(true, false, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, scale, c->w12q + f, 2 * f, nullptr, sms, st);
+    }
+    FP8MLP_TRY(run_quantize_pass(true, true, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, scale, c->w12q, 2 * f, a_w2, sms, st));
+    return run_quantize_pass(true, true, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, scale, c->w12q + f, 2 * f, a_w1, sms, st);
 }
 
 // G|U = Xq [W2q|W1q] with the SwiGLU / Smooth-SwiGLU epilogue
@@ -138,6 +185,9 @@ int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_
     fp8mlp_ctx* c = new (std::nothrow) fp8mlp_ctx();
     if (c == nullptr) return FP8MLP_ERR_ARG;
     std::memset(c, 0, sizeof(*c));
+    c->brackets = new (std::nothrow) std::vector<fp8mlp_ctx::Bracket>();
+    c->free_events = new (std::nothrow) std::vector<cudaEvent_t>();
+    if (c->brackets == nullptr || c->free_events == nullptr) { fp8mlp_destroy(c); return FP8MLP_ERR_ARG; }
     c->T_max = T_max; c->d = d; c->f = f; c->flags = flags; c->saved_T = -1;
     cudaError_t e = cudaGetDevice(&c->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
@@ -170,6 +220,14 @@ int fp8mlp_destroy(fp8mlp_ctx* c) {
     void* ptrs[] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq, c->inv_s, c->dummy, c->status};
     for (void* p : ptrs)
         if (p != nullptr) cudaFree(p);
+    if (c->brackets != nullptr) {
+        for (auto& b : *c->brackets) { cudaEventDestroy(b.e0); cudaEventDestroy(b.e1); }
+        delete c->brackets;
+    }
+    if (c->free_events != nullptr) {
+        for (cudaEvent_t e : *c->free_events) cudaEventDestroy(e);
+        delete c->free_events;
+    }
     delete c;
     return FP8MLP_OK;
 }
@@ -184,6 +242,28 @@ int fp8mlp_status(fp8mlp_ctx* c, void* stream) {
         FP8MLP_CUDA_CHECK(cudaMemsetAsync(c->status, 0, sizeof(int), st));
         return FP8MLP_ERR_TIMEOUT;
     }
+    return FP8MLP_OK;
+}
+
+int fp8mlp_profile_enable(fp8mlp_ctx* c, int on) {
+    if (c == nullptr) return FP8MLP_ERR_ARG;
+    c->profiling = on != 0;
+    return FP8MLP_OK;
+}
+
+int fp8mlp_profile_read(fp8mlp_ctx* c, double* ms, int64_t* count) {
+    if (c == nullptr || ms == nullptr || count == nullptr) return FP8MLP_ERR_ARG;
+    for (int i = 0; i < FP8MLP_PH_COUNT; ++i) { ms[i] = 0.0; count[i] = 0; }
+    for (auto& b : *c->brackets) {
+        FP8MLP_CUDA_CHECK(cudaEventSynchronize(b.e1));
+        float t = 0.0f;
+        FP8MLP_CUDA_CHECK(cudaEventElapsedTime(&t, b.e0, b.e1));
+        ms[b.phase] += t;
+        count[b.phase] += 1;
+        c->free_events->push_back(b.e0);
+        c->free_events->push_back(b.e1);
+    }
+    c->brackets->clear();
     return FP8MLP_OK;
 }
 
@@ -250,41 +330,46 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
     float* a_h = (am && am->h) ? am->h : c->dummy + 8;
     c->saved_T = -1;
 
-    FP8MLP_TRY(zero_floats({a_x, a_w1, a_w2, a_w3}, st));
-    FP8MLP_CUDA_CHECK(cudaMemsetAsync(a_h, 0, sizeof(float) * f, st));
-
-    // x -> E4M3
-    FP8MLP_TRY(quantize_tensor(x, FP8MLP_BF16, T, d, FP8MLP_E4M3, mode, sc->x, a_x, nullptr, nullptr, c->xq, d, c->sm_count, st));
-    // [W2 | W1] -> E4M3 with one scale
-    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
-        FP8MLP_TRY(run_quantize_pass(false, true, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, nullptr, nullptr, 0, a_w1, c->sm_count, st));
-        FP8MLP_TRY(run_quantize_pass(false, true, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, nullptr, nullptr, 0, a_w2, c->sm_count, st));
-        FP8MLP_TRY(run_scale_from_amax(FP8MLP_E4M3, a_w1, a_w2, sc->w12, st));
-        FP8MLP_TRY(run_quantize_pass(true, false, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, sc->w12, c->w12q, 2 * f, nullptr, c->sm_count, st));
-        FP8MLP_TRY(run_quantize_pass(true, false, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, sc->w12, c->w12q + f, 2 * f, nullptr, c->sm_count, st));
-    } else {
-        FP8MLP_TRY(run_quantize_pass(true, true, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, sc->w12, c->w12q, 2 * f, a_w2, c->sm_count, st));
-        FP8MLP_TRY(run_quantize_pass(true, true, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, sc->w12, c->w12q + f, 2 * f, a_w1, c->sm_count, st));
+    {
+        PhaseTimer pt(c, FP8MLP_PH_MISC, st);
+        FP8MLP_TRY(zero_floats({a_x, a_w1, a_w2, a_w3}, st));
+        FP8MLP_CUDA_CHECK(cudaMemsetAsync(a_h, 0, sizeof(float) * f, st));
+    }
+    {   // x -> E4M3
+        PhaseTimer pt(c, FP8MLP_PH_QUANT_X, st);
+        FP8MLP_TRY(quantize_tensor(x, FP8MLP_BF16, T, d, FP8MLP_E4M3, mode, sc->x, a_x, nullptr, nullptr, c->xq, d, c->sm_count, st));
+    }
+    {   // [W2 | W1] -> E4M3 with one scale
+        PhaseTimer pt(c, FP8MLP_PH_QUANT_W12, st);
+        FP8MLP_TRY(quantize_w12(c, W1, W2, mode, sc->w12, a_w1, a_w2, st));
     }
     if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
         // calibration pass: per-channel maxima of H, then s_i (or the per-tensor scale)
-        if (T > 0) FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/0, st));
+        if (T > 0) {
+            PhaseTimer pt(c, FP8MLP_PH_GEMM1, st);
+            FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/0, st));
+        }
+        PhaseTimer pt(c, FP8MLP_PH_MISC, st);
         UpdateScalesArgs u{};
         u.amax_h = a_h; u.scale_h = sc->h; u.f = f; u.smooth = smooth ? 1 : 0;
         FP8MLP_TRY(run_update_scales(u, c->sm_count, st));
     }
-    // W3' = diag(1/s) W3 -> E4M3
-    const float* row_mul = nullptr;
-    if (smooth) {
-        FP8MLP_TRY(run_reciprocal(sc->h, c->inv_s, f, st));
-        row_mul = c->inv_s;
+    {   // W3' = diag(1/s) W3 -> E4M3
+        PhaseTimer pt(c, FP8MLP_PH_QUANT_W3, st);
+        const float* row_mul = nullptr;
+        if (smooth) {
+            FP8MLP_TRY(run_reciprocal(sc->h, c->inv_s, f, st));
+            row_mul = c->inv_s;
+        }
+        FP8MLP_TRY(quantize_tensor(W3, FP8MLP_F32, f, d, FP8MLP_E4M3, mode, sc->w3, a_w3, nullptr, row_mul, c->w3q, d, c->sm_count, st));
     }
-    FP8MLP_TRY(quantize_tensor(W3, FP8MLP_F32, f, d, FP8MLP_E4M3, mode, sc->w3, a_w3, nullptr, row_mul, c->w3q, d, c->sm_count, st));
     if (T == 0) { c->saved_T = (c->flags & FP8MLP_SAVE_FOR_BWD) ? 0 : -1; return FP8MLP_OK; }
-
-    FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/1, st));
-
+    {
+        PhaseTimer pt(c, FP8MLP_PH_GEMM1, st);
+        FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/1, st));
+    }
     // Y = Hq W3q
+    PhaseTimer pt2(c, FP8MLP_PH_GEMM2, st);
     CUtensorMap tmA, tmB;
     FP8MLP_TRY(make_tmap_u8(&tmA, c->hq, f, T, f));
     FP8MLP_TRY(make_tmap_u8(&tmB, c->w3q, d, f, d));
@@ -313,7 +398,10 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
     const int64_t d = c->d, f = c->f;
     float* a_dy = (am && am->dy) ? am->dy : c->dummy + 4;
     float* a_dz = (am && am->dz) ? am->dz : c->dummy + 5;
-    FP8MLP_TRY(zero_floats({a_dy, a_dz}, st));
+    {
+        PhaseTimer pt(c, FP8MLP_PH_MISC, st);
+        FP8MLP_TRY(zero_floats({a_dy, a_dz}, st));
+    }
     if (T == 0) {   // empty batch: the weight gradients are sums over no tokens
         FP8MLP_CUDA_CHECK(cudaMemsetAsync(dW1, 0, sizeof(float) * d * f, st));
         FP8MLP_CUDA_CHECK(cudaMemsetAsync(dW2, 0, sizeof(float) * d * f, st));
@@ -322,8 +410,10 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
     }
     const int Ti = static_cast<int>(T), di = static_cast<int>(d), fi = static_cast<int>(f);
 
-    // dY -> E5M2
-    FP8MLP_TRY(quantize_tensor(dy, FP8MLP_BF16, T, d, FP8MLP_E5M2, mode, sc->dy, a_dy, nullptr, nullptr, c->dyq, d, c->sm_count, st));
+    {   // dY -> E5M2
+        PhaseTimer pt(c, FP8MLP_PH_QUANT_DY, st);
+        FP8MLP_TRY(quantize_tensor(dy, FP8MLP_BF16, T, d, FP8MLP_E5M2, mode, sc->dy, a_dy, nullptr, nullptr, c->dyq, d, c->sm_count, st));
+    }
 
     // dH~ = dYq W3q^T with the SwiGLU-backward epilogue -> dZq = [dG | dU]
     {
@@ -337,12 +427,17 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
         a.amax_dz = reinterpret_cast<unsigned int*>(a_dz);
         if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
             a.store = 0;
-            FP8MLP_TRY(launch_gemm(EPI_SWIGLU_BWD, false, false, FP8MLP_E5M2, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
+            {
+                PhaseTimer pt(c, FP8MLP_PH_DGRAD2, st);
+                FP8MLP_TRY(launch_gemm(EPI_SWIGLU_BWD, false, false, FP8MLP_E5M2, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
+            }
+            PhaseTimer pt(c, FP8MLP_PH_MISC, st);
             UpdateScalesArgs u{};
             u.amax_dz = a_dz; u.scale_dz = sc->dz;
             FP8MLP_TRY(run_update_scales(u, c->sm_count, st));
             a.store = 1;
         }
+        PhaseTimer pt(c, FP8MLP_PH_DGRAD2, st);
         FP8MLP_TRY(launch_gemm(EPI_SWIGLU_BWD, false, false, FP8MLP_E5M2, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
     }
     // dW3 = diag(1/s) (Hq^T dYq)
@@ -353,6 +448,7 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
         GemmArgs a = base_args(c, fi, di, Ti);
         a.s0 = sc->dy; a.row_s = sc->h;
         a.out_f32_0 = dW3; a.out_f32_1 = dW3;
+        PhaseTimer pt(c, FP8MLP_PH_WGRAD3, st);
         FP8MLP_TRY(launch_gemm(EPI_F32, true, true, FP8MLP_E4M3, FP8MLP_E5M2, tmA, tmB, tmB, a, c->sm_count, st));
     }
     // dX = dZq [W2q|W1q]^T
@@ -363,6 +459,7 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
         GemmArgs a = base_args(c, Ti, di, 2 * fi);
         a.s0 = sc->dz; a.s1 = sc->w12;
         a.out_bf16 = static_cast<uint16_t*>(dx);
+        PhaseTimer pt(c, FP8MLP_PH_DGRAD1, st);
         FP8MLP_TRY(launch_gemm(EPI_BF16, false, false, FP8MLP_E5M2, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
     }
     // [dW2 | dW1] = Xq^T dZq
@@ -374,6 +471,7 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
         a.s0 = sc->x; a.s1 = sc->dz;
         a.out_f32_0 = dW2; a.out_f32_1 = dW1;
         a.n_split = fi; a.ld_out = f;
+        PhaseTimer pt(c, FP8MLP_PH_WGRAD12, st);
         FP8MLP_TRY(launch_gemm(EPI_F32, true, true, FP8MLP_E4M3, FP8MLP_E5M2, tmA, tmB, tmB, a, c->sm_count, st));
     }
     return FP8MLP_OK;

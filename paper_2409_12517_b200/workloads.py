@@ -49,16 +49,30 @@ def raw_bits(seed: int, stream: int, start: int, count: int) -> np.ndarray:
         return _mix(_key(seed, stream) + n * _GOLDEN)
 
 
-def normals(seed: int, stream: int, count: int, std: float = 1.0, chunk: int = 1 << 22) -> np.ndarray:
-    """count normal deviates N(0, std^2) as float32 (Box-Muller on 24-bit uniforms)."""
+def _normals_chunk(seed: int, stream: int, lo: int, c: int, std: float, out: np.ndarray) -> None:
+    r = raw_bits(seed, stream, lo, c)
+    u1 = ((r >> np.uint64(40)).astype(np.float64) + 1.0) * (1.0 / 16777216.0)  # (0, 1]
+    u2 = ((r >> np.uint64(8)) & np.uint64(0xFFFFFF)).astype(np.float64) * (1.0 / 16777216.0)
+    z = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+    out[lo:lo + c] = (z * std).astype(np.float32)
+
+
+def normals(seed: int, stream: int, count: int, std: float = 1.0, chunk: int = 1 << 20) -> np.ndarray:
+    """count normal deviates N(0, std^2) as float32 (Box-Muller on 24-bit uniforms).
+
+    Chunks are independent (counter-based), so large draws are spread over host threads;
+    the result does not depend on the number of threads.
+    """
     out = np.empty(count, dtype=np.float32)
-    for lo in range(0, count, chunk):
-        c = min(chunk, count - lo)
-        r = raw_bits(seed, stream, lo, c)
-        u1 = ((r >> np.uint64(40)).astype(np.float64) + 1.0) * (1.0 / 16777216.0)  # (0, 1]
-        u2 = ((r >> np.uint64(8)) & np.uint64(0xFFFFFF)).astype(np.float64) * (1.0 / 16777216.0)
-        z = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
-        out[lo:lo + c] = (z * std).astype(np.float32)
+    starts = list(range(0, count, chunk))
+    if len(starts) <= 2:
+        for lo in starts:
+            _normals_chunk(seed, stream, lo, min(chunk, count - lo), std, out)
+        return out
+    from concurrent.futures import ThreadPoolExecutor
+    import os
+    with ThreadPoolExecutor(max_workers=min(32, os.cpu_count() or 1)) as pool:
+        list(pool.map(lambda lo: _normals_chunk(seed, stream, lo, min(chunk, count - lo), std, out), starts))
     return out
 
 
