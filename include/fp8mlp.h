@@ -46,7 +46,8 @@ enum {
     FP8MLP_ERR_ALIGN = -3,   /* a tensor pointer is not 16-byte aligned                         */
     FP8MLP_ERR_CUDA = -4,    /* a CUDA runtime/driver call failed (see fp8mlp_last_cuda_error)  */
     FP8MLP_ERR_TIMEOUT = -5, /* a kernel gave up on a bounded wait (device status word)         */
-    FP8MLP_ERR_STATE = -6    /* backward without a matching forward that saved activations      */
+    FP8MLP_ERR_STATE = -6,   /* backward without a matching forward that saved activations      */
+    FP8MLP_ERR_TOO_LARGE = -7 /* fp8mlp_forward_static: the problem does not fit the built-in scratch */
 };
 enum { FP8MLP_E4M3 = 0, FP8MLP_E5M2 = 1 };
 enum { FP8MLP_BF16 = 0, FP8MLP_F32 = 1 };
@@ -166,6 +167,37 @@ FP8MLP_API int fp8mlp_forward(fp8mlp_ctx* ctx, int64_t T, const void* x_bf16,
 FP8MLP_API int fp8mlp_backward(fp8mlp_ctx* ctx, int64_t T, const void* dy_bf16,
                     int scale_mode, fp8mlp_scales* scales, fp8mlp_amax* amax,
                     void* dx_bf16, float* dW1, float* dW2, float* dW3, void* stream);
+
+/* Forward without any allocation (the paper has no counterpart; this is a deployment aid).
+ *
+ * Some callers cannot create a context because they cannot allocate device memory at all: a plug-in
+ * running inside a host application whose own pool already owns the whole GPU (cudaMalloc would
+ * fail or fight that pool), or a serving loop that must not hit the device-wide synchronisation
+ * and unpredictable latency a cudaMalloc / cudaFree can bring.  For them this entry point runs the
+ * same forward as fp8mlp_forward (same kernels, forward only, nothing saved for backward) with the
+ * internal buffers - the FP8 copies of x, [W2|W1], W3', the SwiGLU codes, 1/s and the status word -
+ * placed in a fixed array that is part of the library image:
+ *   FP8MLP_STATIC_SCRATCH_BYTES (4 MiB) of device memory, held by every GPU that loads the library
+ *   until the process exits.  The problem fits when
+ *       T*d + 3*d*f + T*f + 8*f + 4096 <= FP8MLP_STATIC_SCRATCH_BYTES
+ *   (e.g. T=128, d=256, f=704, or T=256, d=512, f=1536); otherwise FP8MLP_ERR_TOO_LARGE is returned and
+ *   nothing is launched.
+ * Arguments are those of fp8mlp_forward, with the shape and `flags` (FP8MLP_SMOOTH or 0) passed
+ * directly instead of a context.  The caller still owns x, the weights, y, `scales` and `amax`.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps whatever the previous call left in it; each call
+ *     rewrites or clears everything it reads (the status word and the maxima start from zero).
+ *     Two calls that overlap on the GPU (different streams, or different host threads without
+ *     ordering) race on it: serialise them.
+ *   - A bounded-wait timeout inside a kernel cannot be reported through a context here; the word is
+ *     cleared at the start of every call and is not readable by the caller. */
+#define FP8MLP_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+FP8MLP_API int fp8mlp_forward_static(int64_t T, int64_t d_model, int64_t d_ff, uint32_t flags,
+                                     const void* x_bf16, const float* W1, const float* W2, const float* W3,
+                                     int scale_mode, fp8mlp_scales* scales, fp8mlp_amax* amax,
+                                     void* y_bf16, void* stream);
 
 /* One FP8 GEMM of the kind the block is made of, exposed for tests and tuning (Section 6.2:
  * quantised operands, high-precision accumulation and output).

@@ -15,7 +15,8 @@ import torch
 _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libfp8mlp.so"
 
-OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_CUDA, ERR_TIMEOUT, ERR_STATE = 0, -1, -2, -3, -4, -5, -6
+OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_CUDA, ERR_TIMEOUT, ERR_STATE, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 E4M3, E5M2 = 0, 1
 BF16, F32 = 0, 1
 SMOOTH, SAVE_FOR_BWD = 1, 2
@@ -26,6 +27,7 @@ EXPORTS = [
     "fp8mlp_create", "fp8mlp_destroy", "fp8mlp_strerror", "fp8mlp_last_cuda_error", "fp8mlp_status",
     "fp8mlp_workspace", "fp8mlp_launch_count", "fp8mlp_quantize", "fp8mlp_update_scales",
     "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8", "fp8mlp_profile_enable", "fp8mlp_profile_read",
+    "fp8mlp_forward_static",
 ]
 PHASES = ["quant_x", "quant_w12", "quant_w3", "gemm1_swiglu", "gemm2_down", "quant_dy", "dgrad2_swiglu_bwd",
           "wgrad3", "dgrad1", "wgrad12", "misc"]
@@ -75,6 +77,9 @@ def lib():
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.fp8mlp_gemm_fp8.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int,
                                       C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.fp8mlp_forward_static.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_uint32, C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_int, C.POINTER(_Scales), C.POINTER(_Amax),
+                                            C.c_void_p, C.c_void_p]
         L.fp8mlp_profile_enable.argtypes = [C.c_void_p, C.c_int]
         L.fp8mlp_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         missing = [name for name in EXPORTS if not hasattr(L, name)]
@@ -167,6 +172,16 @@ def fp8mlp_forward(ctx: int, T: int, x, W1, W2, W3, scale_mode: int, scales: dic
     s, a = _scales(scales), _amax(amax)
     _check(lib().fp8mlp_forward(C.c_void_p(ctx), T, _ptr(x), _ptr(W1), _ptr(W2), _ptr(W3), scale_mode, C.byref(s),
                                 C.byref(a) if a is not None else None, _ptr(y), _stream()), "fp8mlp_forward")
+
+
+def fp8mlp_forward_static(T: int, d_model: int, d_ff: int, flags: int, x, W1, W2, W3, scale_mode: int,
+                          scales: dict, amax: dict | None, y) -> None:
+    """Forward for callers that cannot allocate device memory: no context, the library's built-in
+    4 MiB scratch instead (shapes beyond it raise ERR_TOO_LARGE).  Calls that overlap on the GPU race."""
+    s, a = _scales(scales), _amax(amax)
+    _check(lib().fp8mlp_forward_static(T, d_model, d_ff, flags, _ptr(x), _ptr(W1), _ptr(W2), _ptr(W3), scale_mode,
+                                       C.byref(s), C.byref(a) if a is not None else None, _ptr(y), _stream()),
+           "fp8mlp_forward_static")
 
 
 def fp8mlp_backward(ctx: int, T: int, dy, scale_mode: int, scales: dict, amax: dict | None, dx, dW1, dW2, dW3) -> None:

@@ -168,6 +168,7 @@ const char* fp8mlp_strerror(int code) {
         case FP8MLP_ERR_CUDA: return "CUDA call failed";
         case FP8MLP_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
         case FP8MLP_ERR_STATE: return "backward without a matching forward that saved activations";
+        case FP8MLP_ERR_TOO_LARGE: return "problem does not fit the library's built-in scratch (see FP8MLP_STATIC_SCRATCH_BYTES)";
         default: return "unknown error code";
     }
 }
@@ -475,6 +476,60 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
         FP8MLP_TRY(launch_gemm(EPI_F32, true, true, FP8MLP_E4M3, FP8MLP_E5M2, tmA, tmB, tmB, a, c->sm_count, st));
     }
     return FP8MLP_OK;
+}
+
+// ---------------------------------------------------------------- forward without allocation
+}  // extern "C"
+
+namespace {
+// Built-in scratch of fp8mlp_forward_static.  In host code this name is only a stand-in for the
+// symbol: the device address is looked up once per device with cudaGetSymbolAddress.
+__device__ __align__(256) unsigned char g_static_scratch[FP8MLP_STATIC_SCRATCH_BYTES];
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_scratch_ptr[kMaxDevices] = {};   // per device, filled on first use
+
+int64_t round_up_256(int64_t v) { return (v + 255) & ~int64_t(255); }
+}  // namespace
+
+extern "C" {
+
+int fp8mlp_forward_static(int64_t T, int64_t d, int64_t f, uint32_t flags, const void* x, const float* W1,
+                          const float* W2, const float* W3, int mode, fp8mlp_scales* sc, fp8mlp_amax* am, void* y,
+                          void* stream) {
+    if (flags & ~uint32_t(FP8MLP_SMOOTH)) return FP8MLP_ERR_ARG;
+    if (T < 0 || d <= 0 || f <= 0 || d % 16 != 0 || f % 16 != 0) return FP8MLP_ERR_SHAPE;
+    if (T > (1 << 22) || d > (1 << 22) || f > (1 << 22)) return FP8MLP_ERR_TOO_LARGE;
+    if (T * d + 3 * d * f + T * f + 8 * f + 4096 > int64_t(FP8MLP_STATIC_SCRATCH_BYTES)) return FP8MLP_ERR_TOO_LARGE;
+
+    int dev = 0, sms = 0;
+    FP8MLP_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return FP8MLP_ERR_ARG;
+    if (g_static_scratch_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        FP8MLP_CUDA_CHECK(cudaGetSymbolAddress(&p, g_static_scratch));
+        g_static_scratch_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    FP8MLP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+
+    // a context that lives on this stack frame and points into the built-in array
+    fp8mlp_ctx c;
+    std::memset(&c, 0, sizeof(c));
+    c.T_max = T; c.d = d; c.f = f; c.flags = flags; c.device = dev; c.sm_count = sms; c.saved_T = -1;
+    unsigned char* base = g_static_scratch_ptr[dev];
+    int64_t off = 0;
+    auto carve = [&](int64_t bytes) { unsigned char* p = base + off; off += round_up_256(bytes); return p; };
+    c.status = reinterpret_cast<int*>(carve(256));
+    c.dummy = reinterpret_cast<float*>(carve(sizeof(float) * (8 + f)));
+    c.inv_s = reinterpret_cast<float*>(carve(sizeof(float) * f));
+    c.xq = carve(T * d);
+    c.w12q = carve(2 * d * f);
+    c.w3q = carve(f * d);
+    c.hq = carve(T * f);
+    if (off > int64_t(FP8MLP_STATIC_SCRATCH_BYTES)) return FP8MLP_ERR_TOO_LARGE;
+    // the array keeps the previous call's contents: the status word must start at zero (forward
+    // itself clears the maxima it accumulates into)
+    FP8MLP_CUDA_CHECK(cudaMemsetAsync(c.status, 0, sizeof(int), static_cast<cudaStream_t>(stream)));
+    return fp8mlp_forward(&c, T, x, W1, W2, W3, mode, sc, am, y, stream);
 }
 
 int fp8mlp_gemm_fp8(int64_t M, int64_t N, int64_t K, const uint8_t* A, int a_kmajor, int a_fmt, const uint8_t* B,
