@@ -80,9 +80,21 @@ __device__ __forceinline__ float warp_max_nonneg(float v) {
     return __uint_as_float(r);
 }
 
-// sigma(z) = 1 / (1 + e^-z) in fp32
+// sigma(z) = 1 / (1 + e^-z) in fp32 on the special-function unit: 2^x and 1/x to about 2^-22
+// relative, which moves a later FP8 code by one step only where the exact value sits that close
+// to a rounding boundary.  e^-z overflowing to +inf gives 0, underflowing gives 1.
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ float sigmoid_f32(float z) {
-    return __frcp_rn(__fadd_rn(1.0f, expf(-z)));
+    return rcp_approx(__fadd_rn(1.0f, ex2_approx(__fmul_rn(z, -1.4426950408889634f))));
 }
 
 // ---------------------------------------------------------------- mbarrier
@@ -190,6 +202,16 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 // ---------------------------------------------------------------- global memory vectors
 __device__ __forceinline__ void st_global_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// 256-bit accesses (sm_100): the address must be 32-byte aligned
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
+__device__ __forceinline__ void ld_global_nc_v8(const void* p, uint32_t (&w)[8]) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p));
 }
 __device__ __forceinline__ uint4 ld_global_nc_v4(const void* p) {
     uint4 v;

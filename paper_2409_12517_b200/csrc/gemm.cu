@@ -65,178 +65,231 @@ __device__ __forceinline__ bool epi_all(bool v) {
 
 __device__ __forceinline__ float inv_or_one(const float* s) { return s ? __fdiv_rn(1.0f, *s) : 1.0f; }
 
-// ---------------------------------------------------------------- epilogues (one thread = one row)
-__device__ __forceinline__ void epilogue_f32(const GemmArgs& p, uint32_t taddr, int m, int n0, float dq) {
-    const bool row_ok = m < p.M;
-#pragma unroll 1
-    for (int j = 0; j < kBlockN / 32; ++j) {
-        const int c0 = n0 + 32 * j;
-        if (c0 >= p.N) break;
-        uint32_t r[32];
-        tmem_ld32(taddr + 32 * j, r);
-        tmem_ld_wait();
-        if (!row_ok) continue;
+// ---------------------------------------------------------------- epilogues
+// Eight warps drain an accumulator: warp (quad, half) owns TMEM lanes [32 quad, 32 quad + 32) - one
+// row per thread - and one half of the tile's columns, in chunks of 32.  Every chunk is worked
+// through in stages over all 32 elements (independent instructions back to back), and a thread's
+// 32 consecutive outputs leave as whole 32-byte sectors when the rows are 32-byte aligned (wide).
+
+// 32 fp32 values of one row -> global, columns [c0, c0 + 32) of an N-column matrix, 8 at a time
+__device__ __forceinline__ void store_f32x32(const GemmArgs& p, const float (&v)[32], int m, int c0) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int col = c0 + 4 * q;
-            if (col < p.N) {
-                float* dst = col < p.n_split ? p.out_f32_0 + static_cast<int64_t>(m) * p.ld_out + col
-                                             : p.out_f32_1 + static_cast<int64_t>(m) * p.ld_out + (col - p.n_split);
-                st_global_v4(dst, __float_as_uint(__fmul_rn(__uint_as_float(r[4 * q + 0]), dq)),
-                             __float_as_uint(__fmul_rn(__uint_as_float(r[4 * q + 1]), dq)),
-                             __float_as_uint(__fmul_rn(__uint_as_float(r[4 * q + 2]), dq)),
-                             __float_as_uint(__fmul_rn(__uint_as_float(r[4 * q + 3]), dq)));
+    for (int q = 0; q < 4; ++q) {
+        const int col = c0 + 8 * q;
+        if (col < p.N) {
+            float* dst = col < p.n_split ? p.out_f32_0 + static_cast<int64_t>(m) * p.ld_out + col
+                                         : p.out_f32_1 + static_cast<int64_t>(m) * p.ld_out + (col - p.n_split);
+            uint32_t w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) w[e] = __float_as_uint(v[8 * q + e]);
+            if (p.wide) {
+                st_global_v8(dst, w);
+            } else {
+                st_global_v4(dst, w[0], w[1], w[2], w[3]);
+                st_global_v4(dst + 4, w[4], w[5], w[6], w[7]);
             }
         }
     }
 }
 
-__device__ __forceinline__ void epilogue_bf16(const GemmArgs& p, uint32_t taddr, int m, int n0, float dq) {
+__device__ __forceinline__ void epilogue_f32(const GemmArgs& p, uint32_t taddr, int half, int m, int n0, float dq) {
     const bool row_ok = m < p.M;
 #pragma unroll 1
-    for (int j = 0; j < kBlockN / 32; ++j) {
+    for (int jj = 0; jj < 4; ++jj) {
+        const int j = 4 * half + jj;
         const int c0 = n0 + 32 * j;
         if (c0 >= p.N) break;
         uint32_t r[32];
         tmem_ld32(taddr + 32 * j, r);
         tmem_ld_wait();
         if (!row_ok) continue;
+        float v[32];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int col = c0 + 8 * q;
-            if (col < p.N) {
-                uint32_t w[4];
+        for (int e = 0; e < 32; ++e) v[e] = __fmul_rn(__uint_as_float(r[e]), dq);
+        store_f32x32(p, v, m, c0);
+    }
+}
+
+// 16 floats -> 16 bf16 (32 bytes) at dst, columns guarded by the caller
+__device__ __forceinline__ void store_bf16x16(uint16_t* dst, const float* v, bool wide) {
+    uint32_t w[8];
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    w[e] = cvt_bf16x2(__fmul_rn(__uint_as_float(r[8 * q + 2 * e]), dq),
-                                      __fmul_rn(__uint_as_float(r[8 * q + 2 * e + 1]), dq));
-                st_global_v4(p.out_bf16 + static_cast<int64_t>(m) * p.ld_out + col, w[0], w[1], w[2], w[3]);
-            }
-        }
+    for (int e = 0; e < 8; ++e) w[e] = cvt_bf16x2(v[2 * e], v[2 * e + 1]);
+    if (wide) {
+        st_global_v8(dst, w);
+    } else {
+        st_global_v4(dst, w[0], w[1], w[2], w[3]);
+        st_global_v4(dst + 8, w[4], w[5], w[6], w[7]);
+    }
+}
+
+__device__ __forceinline__ void epilogue_bf16(const GemmArgs& p, uint32_t taddr, int half, int m, int n0, float dq) {
+    const bool row_ok = m < p.M;
+#pragma unroll 1
+    for (int jj = 0; jj < 4; ++jj) {
+        const int j = 4 * half + jj;
+        const int c0 = n0 + 32 * j;
+        if (c0 >= p.N) break;
+        uint32_t r[32];
+        tmem_ld32(taddr + 32 * j, r);
+        tmem_ld_wait();
+        if (!row_ok) continue;
+        float v[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) v[e] = __fmul_rn(__uint_as_float(r[e]), dq);
+        uint16_t* dst = p.out_bf16 + static_cast<int64_t>(m) * p.ld_out + c0;
+        store_bf16x16(dst, v, p.wide);
+        if (c0 + 16 < p.N) store_bf16x16(dst + 16, v + 16, p.wide);
+    }
+}
+
+// 32 floats -> 32 FP8 codes (32 bytes) at dst; the second 16 only if `both`
+template <int FMT>
+__device__ __forceinline__ void store_fp8x32(uint8_t* dst, const float (&v)[32], bool both, bool wide) {
+    uint32_t w[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) w[e] = cvt_fp8x4<FMT>(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+    if (both && wide) {
+        st_global_v8(dst, w);
+    } else {
+        st_global_v4(dst, w[0], w[1], w[2], w[3]);
+        if (both) st_global_v4(dst + 16, w[4], w[5], w[6], w[7]);
     }
 }
 
 // Forward: accumulator columns [0,128) are G = x W2 (gate), [128,256) are U = x W1 (linear) of the
-// same 128 channels.  H = U * G * sigma(G); per-channel max |H|; Hq = Q_e4m3(H * s_i); bf16 G, U kept
-// for backward.  H itself never leaves the SM.
+// same 128 channels; this warp takes channels [64 half, 64 half + 64) of them.
+// H = U * G * sigma(G); per-channel max |H|; Hq = Q_e4m3(H * s_i); bf16 G, U kept for backward.
+// H itself never leaves the SM.
 __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail* tail, uint32_t taddr, int lane,
-                                                    int m, int n0, float dq) {
+                                                    int half, int m, int n0, float dq) {
     const bool row_ok = m < p.M;
     const int f = p.N;
 #pragma unroll 1
-    for (int j = 0; j < 4; ++j) {
+    for (int jj = 0; jj < 2; ++jj) {
+        const int j = 2 * half + jj;
         const int c0 = n0 + 32 * j;
         if (c0 >= f) break;
         uint32_t g_raw[32], u_raw[32];
         tmem_ld32(taddr + 32 * j, g_raw);
         tmem_ld32(taddr + 128 + 32 * j, u_raw);
         tmem_ld_wait();
-        float hs[32];
+        float g[32], u[32], h[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            g[e] = __fmul_rn(__uint_as_float(g_raw[e]), dq);
+            u[e] = __fmul_rn(__uint_as_float(u_raw[e]), dq);
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) h[e] = ex2_approx(__fmul_rn(g[e], -1.4426950408889634f));
+#pragma unroll
+        for (int e = 0; e < 32; ++e) h[e] = rcp_approx(__fadd_rn(1.0f, h[e]));          // sigma(G)
+#pragma unroll
+        for (int e = 0; e < 32; ++e) h[e] = __fmul_rn(u[e], __fmul_rn(g[e], h[e]));       // H
         float colmax = 0.0f;
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
-            const float g = __fmul_rn(__uint_as_float(g_raw[e]), dq);
-            const float u = __fmul_rn(__uint_as_float(u_raw[e]), dq);
-            const float sw = __fmul_rn(g, sigmoid_f32(g));
-            const float h = __fmul_rn(u, sw);
-            const float cm = warp_max_nonneg(fabsf(h));       // max over this warp's 32 rows
+            const float cm = warp_max_nonneg(fabsf(h[e]));       // max over this warp's 32 rows
             if (lane == e) colmax = cm;
-            hs[e] = __fmul_rn(h, tail->s_tile[0][32 * j + e]);
-            g_raw[e] = __float_as_uint(g);
-            u_raw[e] = __float_as_uint(u);
         }
         atomicMax(&tail->amax_tile[32 * j + lane], __float_as_uint(colmax));
         if (!p.store || !row_ok) continue;
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const int col = c0 + 16 * q;
-            if (col < f) {
-                uint32_t w[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    w[e] = cvt_fp8x4<FP8MLP_E4M3>(hs[16 * q + 4 * e], hs[16 * q + 4 * e + 1], hs[16 * q + 4 * e + 2],
-                                                 hs[16 * q + 4 * e + 3]);
-                st_global_v4(p.hq + static_cast<int64_t>(m) * f + col, w[0], w[1], w[2], w[3]);
-            }
-        }
+        const bool both = c0 + 16 < f;
         if (p.gu != nullptr) {
-            uint16_t* grow = p.gu + static_cast<int64_t>(m) * 2 * f;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int col = c0 + 8 * q;
-                if (col < f) {
-                    uint32_t wg[4], wu[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        wg[e] = cvt_bf16x2(__uint_as_float(g_raw[8 * q + 2 * e]), __uint_as_float(g_raw[8 * q + 2 * e + 1]));
-                        wu[e] = cvt_bf16x2(__uint_as_float(u_raw[8 * q + 2 * e]), __uint_as_float(u_raw[8 * q + 2 * e + 1]));
-                    }
-                    st_global_v4(grow + col, wg[0], wg[1], wg[2], wg[3]);
-                    st_global_v4(grow + f + col, wu[0], wu[1], wu[2], wu[3]);
-                }
+            uint16_t* grow = p.gu + static_cast<int64_t>(m) * 2 * f + c0;
+            store_bf16x16(grow, g, true);
+            store_bf16x16(grow + f, u, true);
+            if (both) {
+                store_bf16x16(grow + 16, g + 16, true);
+                store_bf16x16(grow + f + 16, u + 16, true);
             }
         }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) h[e] = __fmul_rn(h[e], tail->s_tile[0][32 * j + e]);
+        store_fp8x32<FP8MLP_E4M3>(p.hq + static_cast<int64_t>(m) * f + c0, h, both, p.wide);
     }
 }
 
-// Backward: accumulator = dY W3'^T for 256 channels.  dH = acc * dq (* s_i with Smooth-SwiGLU);
-// dU = dH * G sigma(G); dG = dH * U * sigma(G) (1 + G (1 - sigma(G))); max of |dG|, |dU|;
-// dZq = Q_e5m2([dG | dU] * sdz).
-__device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const float* s_tile, uint32_t taddr, int m,
-                                                     int n0, float dq, float sdz) {
+// Saved bf16 G and U of one row, 32 channels each (4 x 32 bytes), for the backward epilogue.
+struct GuChunk { uint32_t g[16], u[16]; };
+__device__ __forceinline__ void load_gu(const GemmArgs& p, int m, int c0, GuChunk& r) {
+    const int f = p.N;
+    const bool lo = m < p.M && c0 < f, hi = m < p.M && c0 + 16 < f;
+    const uint16_t* grow = p.gu + static_cast<int64_t>(m) * 2 * f + c0;
+    uint32_t(&g0)[8] = *reinterpret_cast<uint32_t(*)[8]>(r.g);
+    uint32_t(&g1)[8] = *reinterpret_cast<uint32_t(*)[8]>(r.g + 8);
+    uint32_t(&u0)[8] = *reinterpret_cast<uint32_t(*)[8]>(r.u);
+    uint32_t(&u1)[8] = *reinterpret_cast<uint32_t(*)[8]>(r.u + 8);
+    if (lo) { ld_global_nc_v8(grow, g0); ld_global_nc_v8(grow + f, u0); }
+    else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { g0[e] = 0u; u0[e] = 0u; }
+    }
+    if (hi) { ld_global_nc_v8(grow + 16, g1); ld_global_nc_v8(grow + f + 16, u1); }
+    else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { g1[e] = 0u; u1[e] = 0u; }
+    }
+}
+
+// Backward: accumulator = dY W3'^T for 256 channels; this warp takes [128 half, 128 half + 128).
+// dH = acc * dq (* s_i with Smooth-SwiGLU); dU = dH * G sigma(G);
+// dG = dH * U * sigma(G) (1 + G (1 - sigma(G))); max of |dG|, |dU|; dZq = Q_e5m2([dG | dU] * sdz).
+// `first` holds the saved G, U of the first chunk, requested before the accumulator was ready;
+// each chunk requests the next one's before it starts computing.
+__device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const float* s_tile, uint32_t taddr, int half,
+                                                     int m, int n0, float dq, float sdz, GuChunk& first) {
     const bool row_ok = m < p.M;
     const int f = p.N;
     float local_max = 0.0f;
-#pragma unroll 1
-    for (int j = 0; j < kBlockN / 32; ++j) {
+    GuChunk next;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+        GuChunk& cur = (jj & 1) ? next : first;
+        GuChunk& nxt = (jj & 1) ? first : next;
+        const int j = 4 * half + jj;
         const int c0 = n0 + 32 * j;
         if (c0 >= f) break;
         uint32_t acc[32];
         tmem_ld32(taddr + 32 * j, acc);
-        uint4 gq[4], uq[4];
-        const uint16_t* grow = p.gu + static_cast<int64_t>(m) * 2 * f + c0;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const bool ok = row_ok && (c0 + 8 * q) < f;
-            gq[q] = ok ? ld_global_nc_v4(grow + 8 * q) : make_uint4(0, 0, 0, 0);
-            uq[q] = ok ? ld_global_nc_v4(grow + f + 8 * q) : make_uint4(0, 0, 0, 0);
-        }
+        if (jj < 3) load_gu(p, m, c0 + 32, nxt);
         tmem_ld_wait();
         float dg[32], du[32];
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
-            const uint32_t gw = reinterpret_cast<const uint32_t*>(gq)[e >> 1];
-            const uint32_t uw = reinterpret_cast<const uint32_t*>(uq)[e >> 1];
-            const float g = (e & 1) ? bf16_hi(gw) : bf16_lo(gw);
-            const float u = (e & 1) ? bf16_hi(uw) : bf16_lo(uw);
             float dh = __fmul_rn(__uint_as_float(acc[e]), dq);
             if (p.smooth) dh = __fmul_rn(dh, s_tile[32 * j + e]);
-            const float sig = sigmoid_f32(g);
-            const float sw = __fmul_rn(g, sig);
-            du[e] = __fmul_rn(dh, sw);
+            du[e] = dh;
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const uint32_t gw = cur.g[e >> 1];
+            const float g = (e & 1) ? bf16_hi(gw) : bf16_lo(gw);
+            dg[e] = ex2_approx(__fmul_rn(g, -1.4426950408889634f));
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) dg[e] = rcp_approx(__fadd_rn(1.0f, dg[e]));         // sigma(G)
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const uint32_t gw = cur.g[e >> 1], uw = cur.u[e >> 1];
+            const float g = (e & 1) ? bf16_hi(gw) : bf16_lo(gw);
+            const float u = (e & 1) ? bf16_hi(uw) : bf16_lo(uw);
+            const float dh = du[e], sig = dg[e];
+            du[e] = __fmul_rn(dh, __fmul_rn(g, sig));
             const float t1 = __fadd_rn(1.0f, __fmul_rn(g, __fsub_rn(1.0f, sig)));
-            const float dsw = __fmul_rn(sig, t1);
-            dg[e] = __fmul_rn(__fmul_rn(dh, u), dsw);
+            dg[e] = __fmul_rn(__fmul_rn(dh, u), __fmul_rn(sig, t1));
             local_max = fmaxf(local_max, fmaxf(fabsf(dg[e]), fabsf(du[e])));
         }
         if (!p.store || !row_ok) continue;
-        uint8_t* zrow = p.dzq + static_cast<int64_t>(m) * 2 * f + c0;
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            if (c0 + 16 * q < f) {
-                uint32_t wg[4], wu[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int b = 16 * q + 4 * e;
-                    wg[e] = cvt_fp8x4<FP8MLP_E5M2>(__fmul_rn(dg[b], sdz), __fmul_rn(dg[b + 1], sdz),
-                                                  __fmul_rn(dg[b + 2], sdz), __fmul_rn(dg[b + 3], sdz));
-                    wu[e] = cvt_fp8x4<FP8MLP_E5M2>(__fmul_rn(du[b], sdz), __fmul_rn(du[b + 1], sdz),
-                                                  __fmul_rn(du[b + 2], sdz), __fmul_rn(du[b + 3], sdz));
-                }
-                st_global_v4(zrow + 16 * q, wg[0], wg[1], wg[2], wg[3]);
-                st_global_v4(zrow + f + 16 * q, wu[0], wu[1], wu[2], wu[3]);
-            }
+        for (int e = 0; e < 32; ++e) {
+            dg[e] = __fmul_rn(dg[e], sdz);
+            du[e] = __fmul_rn(du[e], sdz);
         }
+        uint8_t* zrow = p.dzq + static_cast<int64_t>(m) * 2 * f + c0;
+        const bool both = c0 + 16 < f;
+        store_fp8x32<FP8MLP_E5M2>(zrow, dg, both, p.wide);
+        store_fp8x32<FP8MLP_E5M2>(zrow + f, du, both, p.wide);
     }
     return local_max;
 }
@@ -339,9 +392,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------ epilogue (warps 2..9)
         const int quad = warp & 3;                     // TMEM lanes [32*quad, 32*quad+32) belong to this warp
+        const int half = (warp - 2) >> 2;              // which half of the tile's columns
         const int row = quad * 32 + lane;
+        const int et = (warp - 2) * 32 + lane;         // index among the epilogue threads
         const float dq0 = __fmul_rn(inv_or_one(p.s0), inv_or_one(p.s1));
         float sdz = 1.0f;
         if constexpr (EPI == EPI_SWIGLU_BWD) sdz = *p.sdz;
@@ -354,12 +409,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int n0 = n_tile * p.n_tile_cols;
             const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
             if constexpr (EPI == EPI_SWIGLU_FWD) {
-                tail->s_tile[0][row] = (n0 + row) < p.N ? p.s_h[n0 + row] : 1.0f;
-                tail->amax_tile[row] = 0u;
+                if (et < 128) {
+                    tail->s_tile[0][et] = (n0 + et) < p.N ? p.s_h[n0 + et] : 1.0f;
+                    tail->amax_tile[et] = 0u;
+                }
             }
+            GuChunk gu_first;
             if constexpr (EPI == EPI_SWIGLU_BWD) {
-                tail->s_tile[acc][row] = (n0 + row) < p.N ? p.s_h[n0 + row] : 1.0f;
-                tail->s_tile[acc][row + 128] = (n0 + row + 128) < p.N ? p.s_h[n0 + row + 128] : 1.0f;
+                tail->s_tile[acc][et] = (n0 + et) < p.N ? p.s_h[n0 + et] : 1.0f;
+                load_gu(p, m, n0 + 128 * half, gu_first);   // does not depend on the accumulator
             }
             const bool got = mbar_wait(smem_u32(&tail->tmem_full[acc]), acc_phase, abort_flag, p.status);
             if (!epi_all(got)) break;                  // also orders the s_tile / amax_tile writes above
@@ -369,22 +427,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 float dq = dq0;
                 if (p.row_s != nullptr)
                     dq = __fmul_rn(inv_or_one(p.s0), m < p.M ? __fdiv_rn(1.0f, p.row_s[m]) : 1.0f);
-                epilogue_f32(p, taddr, m, n0, dq);
+                epilogue_f32(p, taddr, half, m, n0, dq);
             } else if constexpr (EPI == EPI_BF16) {
-                epilogue_bf16(p, taddr, m, n0, dq0);
+                epilogue_bf16(p, taddr, half, m, n0, dq0);
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
-                epilogue_swiglu_fwd(p, tail, taddr, lane, m, n0, dq0);
+                epilogue_swiglu_fwd(p, tail, taddr, lane, half, m, n0, dq0);
             } else {
-                run_max = fmaxf(run_max, epilogue_swiglu_bwd(p, tail->s_tile[acc], taddr, m, n0, dq0, sdz));
+                run_max = fmaxf(run_max, epilogue_swiglu_bwd(p, tail->s_tile[acc], taddr, half, m, n0, dq0, sdz, gu_first));
             }
             // accumulator drained: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tail->tmem_empty[acc]));
             if constexpr (EPI == EPI_SWIGLU_FWD) {
-                epi_bar_sync();                        // all four row quadrants have merged into amax_tile
-                const unsigned int v = tail->amax_tile[row];
-                if ((n0 + row) < p.N && v != 0u) atomicMax(p.amax_h + n0 + row, v);
+                epi_bar_sync();                        // all eight warps have merged into amax_tile
+                if (et < 128) {
+                    const unsigned int v = tail->amax_tile[et];
+                    if ((n0 + et) < p.N && v != 0u) atomicMax(p.amax_h + n0 + et, v);
+                }
                 // each thread resets only its own amax_tile / s_tile entry for the next tile, and the
                 // others touch them again only after the next tile's barrier: no second barrier needed
             }
@@ -475,6 +535,14 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     args.idesc = (1u << 4) | (static_cast<uint32_t>(a_fmt) << 7) | (static_cast<uint32_t>(b_fmt) << 10) |
                  (static_cast<uint32_t>(a_mn) << 15) | (static_cast<uint32_t>(b_mn) << 16) |
                  (static_cast<uint32_t>(kBlockN >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+    // 32-byte stores need 32-byte aligned rows: the caller's pointers are only promised 16
+    auto al32 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 31u) == 0; };
+    switch (epi) {
+        case EPI_F32: args.wide = al32(args.out_f32_0) && al32(args.out_f32_1); break;
+        case EPI_BF16: args.wide = al32(args.out_bf16); break;
+        case EPI_SWIGLU_FWD: args.wide = al32(args.hq) && args.N % 32 == 0; break;
+        default: args.wide = al32(args.dzq) && args.N % 32 == 0; break;
+    }
     const int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
     if (tiles == 0 || args.num_k_blocks == 0) return FP8MLP_OK;
     const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);

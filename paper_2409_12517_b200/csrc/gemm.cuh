@@ -9,8 +9,8 @@
 // 128-byte swizzle and only the shared-memory matrix descriptors differ.  That lets the forward,
 // dgrad and wgrad GEMMs of the block all read the same FP8 buffers without transposed copies.
 //
-// CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the MMAs,
-// warps 2-5 are the epilogue (one TMEM lane quadrant each).  Two 256-column accumulators
+// CTA = 10 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the MMAs,
+// warps 2-9 are the epilogue (a TMEM lane quadrant and one half of the columns each).  Two 256-column accumulators
 // alternate, so the epilogue of one tile overlaps the main loop of the next.
 // Every wait is bounded: on expiry the CTA raises a status word and drains.
 #pragma once
@@ -28,9 +28,9 @@ constexpr int kUmmaK = 32;            // contraction elements per tcgen05.mma (3
 constexpr int kStages = 4;
 constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 bytes x 128 rows
 constexpr int kStageBytes = 3 * kBoxBytes;   // A box + two B boxes
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 320;
 constexpr int kTmemCols = 512;
-constexpr int kEpiThreads = 128;
+constexpr int kEpiThreads = 256;
 
 struct GemmArgs {
     int M, N, K;            // N: extent of the n coordinate space (output columns; d_ff channels for the SwiGLU epilogues)
@@ -57,6 +57,7 @@ struct GemmArgs {
     const float* s_h;       // [f] per-channel scale of H
     int smooth;             // backward: multiply dH by s_h (Smooth-SwiGLU) or not (per-tensor scale)
     int store;              // 0: calibration pass, only the maxima are produced
+    int wide;               // outputs may be written 32 bytes at a time (rows and bases 32-byte aligned)
     uint8_t* hq;            // fwd: E4M3 [M, f]
     uint16_t* gu;           // fwd: out (nullable), bwd: in; bf16 [M, 2f] = G | U
     unsigned int* amax_h;   // fwd: [f] bit patterns of max |H|, raised atomically
