@@ -37,3 +37,27 @@ def nmax_err(got: np.ndarray, ref: np.ndarray) -> float:
 
 def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def bf16_ulp(v: np.ndarray) -> np.ndarray:
+    """Spacing of bf16 values (8 significant bits) at the magnitude of v."""
+    a = np.abs(v.astype(np.float64))
+    e = np.floor(np.log2(np.maximum(a, 2.0 ** -126)))
+    return 2.0 ** (e - 7)
+
+
+def nmax_err_bf16(got_bits: np.ndarray, ref: np.ndarray) -> float:
+    """Normalised max error of a bf16 output against the oracle's, net of the output rounding:
+    two fp32 results within eps of each other round to bf16 values at most eps + one bf16 spacing
+    apart, so one spacing is granted per element and the rest is held to the bar on eps."""
+    got = bf16_bits_to_f32(got_bits).astype(np.float64)
+    ref = ref.astype(np.float64)
+    excess = np.maximum(np.abs(got - ref) - bf16_ulp(ref), 0.0)
+    denom = np.abs(ref).max()
+    return float(excess.max() / (denom if denom > 0 else 1.0))
+
+
+def frac_beyond(got: np.ndarray, ref: np.ndarray, tol: float) -> float:
+    """Fraction of elements whose error exceeds tol * max |ref|."""
+    ref = ref.astype(np.float64)
+    return float(np.mean(np.abs(got.astype(np.float64) - ref) > tol * np.abs(ref).max()))

@@ -1,0 +1,174 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times
+(Smooth-SwiGLU on, activations saved, delayed scaling: scales given, maxima emitted).
+
+The whole oracle would take hours at these sizes, so the comparison is on sampled outputs the
+oracle computes in full, each with its complete contraction:
+  - everything that is one pass over a tensor (the quantised x, [W2|W1], W3', dY and their maxima)
+    is compared in full, bit for bit;
+  - a sample of tokens gives whole rows of Hq, G, U, Y, dZq and dX (a token's outputs depend on no
+    other token once the scales are given);
+  - a sample of channels - every outlier channel among them - gives whole columns of Hq and dZq,
+    the per-channel maxima, rows of dW3 and columns of dW1, dW2 (a channel's outputs depend on no
+    other channel once the scales are given).
+That a token / channel sub-problem reproduces the rows / columns of the full run is pinned on the
+CPU in test_oracle_pins.py.  The given scales come from an oracle run on a small batch drawn with
+another seed (the "previous iteration" of delayed scaling), never from the CUDA path.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import bf16_bits_to_f32, code_mismatch, frac_beyond, nmax_err, nmax_err_bf16, to_dev, to_dev_bf16
+from paper_2409_12517_b200 import binding as B
+from paper_2409_12517_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+CODE_FRAC = 1e-3
+OUT_TOL = 2e-3
+AMAX_RTOL = 1e-5
+
+
+def _previous_iteration_scales(w, n_tokens):
+    """Scales a delayed-scaling run would hold: from the oracle on a small batch of another seed,
+    with two binades of headroom for the activations (the maxima of a few tokens underestimate those
+    of thousands)."""
+    cfg = dict(wl.CONFIGS[w.name])
+    cfg.update(seed=cfg["seed"] + 100, T=n_tokens)
+    prev = wl.make("prev", **cfg)
+    pf = oracle.forward(prev.x, w.W1, w.W2, w.W3)
+    pb = oracle.backward(pf, prev.dY)
+    s_h = (pf["s_h"] * np.float32(0.25)).astype(np.float32)
+    inv = (np.float32(1.0) / s_h).astype(np.float32)
+    sw3 = oracle.scale_from_amax(oracle.E4M3, oracle.amax(w.W3, inv))
+    return dict(x=np.float32(pf["sx"] * 0.5), w12=np.float32(pf["sw12"]), w3=np.float32(sw3), h=s_h,
+                dy=np.float32(pb["sdy"] * 0.5), dz=np.float32(pb["sdz"] * 0.25))
+
+
+def _check_bf16_rows(name, got_bits, ref):
+    """Y and dX are bf16 roundings of fp32 results.  Where the two fp32 values straddle a rounding
+    boundary the bf16 values are one spacing apart, which on an element above a quarter of the
+    maximum is already more than 2e-3 of it: the bar is applied net of that one spacing, and the
+    elements that need the allowance must be few."""
+    e = nmax_err_bf16(got_bits, ref)
+    assert e <= OUT_TOL, f"{name} rows: {e}"
+    fr = frac_beyond(bf16_bits_to_f32(got_bits), ref, OUT_TOL)
+    assert fr <= 1e-2, f"{name} rows: {fr:.2e} of the elements are a bf16 spacing off"
+
+
+def _check_dz_codes(name, got, ref):
+    """E5M2 codes of [dG | dU].  They inherit the accumulation-order differences like Hq does (one
+    code step, rarely), and one more: the saved bf16 G and U may themselves differ by one bf16
+    spacing between the two sides, and near the zero of the gate derivative (G about -1.28) that
+    moves a small dG by more than one of its own code steps.  So: few codes differ at all, hardly
+    any by more than one step, and every difference is small against the tensor (the bar for
+    gradient values)."""
+    frac, worst = code_mismatch(got, ref)
+    assert frac <= CODE_FRAC, f"{name}: {frac:.2e} of the codes differ"
+    if worst > 1:
+        from helpers import code_rank
+        many = float(np.mean(np.abs(code_rank(got) - code_rank(ref)) > 1))
+        assert many <= 2e-5, f"{name}: {many:.2e} of the codes differ by more than one step"
+        dv, rv = oracle.decode(oracle.E5M2, got), oracle.decode(oracle.E5M2, ref)
+        assert nmax_err(dv, rv) <= OUT_TOL, f"{name}: decoded difference {nmax_err(dv, rv)}"
+
+
+def _sample(rng, n, count, always=()):
+    picks = set(int(i) for i in always)
+    picks.update({0, n - 1, 127, 128, n // 2})
+    while len(picks) < count:
+        picks.add(int(rng.integers(0, n)))
+    return np.array(sorted(picks), dtype=np.int64)
+
+
+@pytest.mark.parametrize("name,n_prev,n_tok,n_ch", [("7b", 48, 24, 32), ("70b", 16, 8, 20)])
+def test_full_size_sampled_parity(name, n_prev, n_tok, n_ch):
+    w = wl.make_config(name)
+    T, d, f = w.T, w.d, w.f
+    given = _previous_iteration_scales(w, n_prev)
+    rng = np.random.default_rng(1234)
+    toks = _sample(rng, T, n_tok, w.outlier_tokens[:4])
+    chans = _sample(rng, f, n_ch, w.outlier_channels)
+
+    # ---- CUDA path: one delayed-scaling step through the C ABI
+    ctx = B.fp8mlp_create(T, d, f, B.SMOOTH | B.SAVE_FOR_BWD)
+    try:
+        sc, am = B.new_scales(f), B.new_amax(f)
+        for k, v in given.items():
+            sc[k].copy_(to_dev(np.atleast_1d(np.asarray(v, np.float32))))
+        W1, W2, W3 = to_dev(w.W1), to_dev(w.W2), to_dev(w.W3)
+        y = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        dx = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        dW1 = torch.full((d, f), float("nan"), device="cuda")
+        dW2 = torch.full((d, f), float("nan"), device="cuda")
+        dW3 = torch.full((f, d), float("nan"), device="cuda")
+        B.fp8mlp_forward(ctx, T, to_dev_bf16(w.x), W1, W2, W3, B.SCALE_GIVEN, sc, am, y)
+        B.fp8mlp_backward(ctx, T, to_dev_bf16(w.dY), B.SCALE_GIVEN, sc, am, dx, dW1, dW2, dW3)
+        assert B.fp8mlp_status(ctx) == B.OK
+        del W1, W2, W3
+        ws = lambda which, shape, dt=torch.uint8: B.workspace_tensor(ctx, which, shape, dt)
+        ti, ci = torch.from_numpy(toks).cuda(), torch.from_numpy(chans).cuda()
+        ci2 = torch.cat([ci, ci + f])
+        got = dict(Xq=ws(B.WS_XQ, (T, d)).cpu().numpy(), W12q=ws(B.WS_W12Q, (d, 2 * f)).cpu().numpy(),
+                   W3q=ws(B.WS_W3Q, (f, d)).cpu().numpy(), dYq=ws(B.WS_DYQ, (T, d)).cpu().numpy())
+        hq, dzq = ws(B.WS_HQ, (T, f)), ws(B.WS_DZQ, (T, 2 * f))
+        gu = ws(B.WS_GU, (T, 2 * f), torch.int16)
+        got.update(Hq_rows=hq[ti].cpu().numpy(), Hq_cols=hq[:, ci].cpu().numpy(),
+                   dZq_rows=dzq[ti].cpu().numpy(), dZq_cols=dzq[:, ci2].cpu().numpy(),
+                   GU_rows=gu[ti].cpu().numpy().view(np.uint16),
+                   Y_rows=y[ti].view(torch.int16).cpu().numpy().view(np.uint16),
+                   dX_rows=dx[ti].view(torch.int16).cpu().numpy().view(np.uint16),
+                   dW1_cols=dW1[:, ci].cpu().numpy(), dW2_cols=dW2[:, ci].cpu().numpy(), dW3_rows=dW3[ci].cpu().numpy())
+        assert bool(torch.isfinite(dW1).all()) and bool(torch.isfinite(dW2).all()) and bool(torch.isfinite(dW3).all())
+        del hq, dzq, gu
+        amax = {k: v.cpu().numpy() for k, v in am.items()}
+        scales = {k: v.cpu().numpy() for k, v in sc.items()}
+    finally:
+        B.fp8mlp_destroy(ctx)
+    for k, v in given.items():                               # given scales are left alone
+        assert np.array_equal(scales[k], np.atleast_1d(np.asarray(v, np.float32)))
+
+    # ---- one-pass tensors, in full, bit for bit
+    x_f = wl.bf16_bits_to_f32(w.x)
+    assert amax["x"][0] == np.float32(oracle.amax(x_f))
+    assert np.array_equal(got["Xq"], oracle.quantize(x_f, oracle.E4M3, given["x"])[0]), "x codes"
+    del x_f
+    assert amax["w1"][0] == np.float32(oracle.amax(w.W1)) and amax["w2"][0] == np.float32(oracle.amax(w.W2))
+    assert np.array_equal(got["W12q"][:, :f], oracle.quantize(w.W2, oracle.E4M3, given["w12"])[0]), "W2 codes"
+    assert np.array_equal(got["W12q"][:, f:], oracle.quantize(w.W1, oracle.E4M3, given["w12"])[0]), "W1 codes"
+    inv_s = (np.float32(1.0) / given["h"]).astype(np.float32)
+    w3q, _, a_w3 = oracle.quantize(w.W3, oracle.E4M3, given["w3"], row_mul=inv_s)
+    assert amax["w3"][0] == np.float32(a_w3) and np.array_equal(got["W3q"], w3q), "W3' codes"
+    dy_f = wl.bf16_bits_to_f32(w.dY)
+    assert amax["dy"][0] == np.float32(oracle.amax(dy_f))
+    assert np.array_equal(got["dYq"], oracle.quantize(dy_f, oracle.E5M2, given["dy"])[0]), "dY codes"
+    del dy_f
+
+    # ---- sampled tokens: whole rows
+    og = dict(scale_mode=oracle.SCALE_GIVEN, sx=float(given["x"]), sw12=float(given["w12"]), s_h=given["h"],
+              sw3=float(given["w3"]))
+    fw = oracle.forward(w.x[toks], w.W1, w.W2, w.W3, **og)
+    bw = oracle.backward(fw, w.dY[toks], scale_mode=oracle.SCALE_GIVEN, sdy=float(given["dy"]), sdz=float(given["dz"]))
+    frac, worst = code_mismatch(got["Hq_rows"], fw["Hq"])
+    assert worst <= 1 and frac <= CODE_FRAC, f"Hq rows: {frac:.2e} differ, worst {worst}"
+    for nm, g_bits, ref in (("G", got["GU_rows"][:, :f], fw["G"]), ("U", got["GU_rows"][:, f:], fw["U"])):
+        assert nmax_err_bf16(g_bits, bf16_bits_to_f32(ref)) <= 1e-5, f"saved {nm}"
+    _check_bf16_rows("Y", got["Y_rows"], fw["Y"])
+    _check_dz_codes("dZq rows", got["dZq_rows"], bw["dZq"])
+    _check_bf16_rows("dX", got["dX_rows"], bw["dX"])
+    assert amax["dz"][0] >= 0.999 * bw["amax_dz"]            # the global maximum covers the sample's
+    del fw, bw
+
+    # ---- sampled channels: whole columns, per-channel maxima, weight-gradient slices
+    ogc = dict(og, s_h=given["h"][chans])
+    fwc = oracle.forward(w.x, w.W1[:, chans], w.W2[:, chans], w.W3[chans, :], **ogc)
+    bwc = oracle.backward(fwc, w.dY, scale_mode=oracle.SCALE_GIVEN, sdy=float(given["dy"]), sdz=float(given["dz"]))
+    assert np.allclose(amax["h"][chans], fwc["amax_h"], rtol=AMAX_RTOL, atol=0), "per-channel maxima of H"
+    frac, worst = code_mismatch(got["Hq_cols"], fwc["Hq"])
+    assert worst <= 1 and frac <= CODE_FRAC, f"Hq columns: {frac:.2e} differ, worst {worst}"
+    _check_dz_codes("dZq columns", got["dZq_cols"], bwc["dZq"])
+    for nm, g, ref in (("dW1", got["dW1_cols"], bwc["dW1"]), ("dW2", got["dW2_cols"], bwc["dW2"]),
+                       ("dW3", got["dW3_rows"], bwc["dW3"])):
+        e = nmax_err(g, ref)
+        assert e <= OUT_TOL, f"{nm} slices: {e}"
