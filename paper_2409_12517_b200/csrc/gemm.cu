@@ -8,17 +8,27 @@ namespace fp8mlp {
 namespace {
 
 // ---------------------------------------------------------------- shared memory plan
+// Single CTA: a stage holds an A box and two B boxes (128 x 256 tile).  CTA pair: a stage holds this
+// CTA's A box and its one B box (its halves of a 256 x 256 tile).
+template <bool PAIR> struct Plan;
+template <> struct Plan<false> { static constexpr int kStages = 4, kStageBytes = 3 * kBoxBytes, kTileM = 128; };
+template <> struct Plan<true>  { static constexpr int kStages = 6, kStageBytes = 2 * kBoxBytes, kTileM = 256; };
+constexpr int kMaxStages = 6;
+
 struct __align__(8) SmemTail {
-    uint64_t full[kStages];      // TMA -> MMA: stage filled
-    uint64_t empty[kStages];     // MMA -> TMA: stage drained
+    uint64_t full[kMaxStages];   // TMA -> MMA: stage filled (CTA pair: only rank 0's are used)
+    uint64_t empty[kMaxStages];  // MMA -> TMA: stage drained
     uint64_t tmem_full[2];       // MMA -> epilogue: accumulator complete
-    uint64_t tmem_empty[2];      // epilogue -> MMA: accumulator drained
+    uint64_t tmem_empty[2];      // epilogue -> MMA: accumulator drained (CTA pair: rank 0's count both CTAs)
     uint32_t tmem_base;
     int abort;
     float s_tile[2][kBlockN];    // per-channel scales of the current tile(s)
     unsigned int amax_tile[128]; // per-channel maxima of the current tile (forward)
 };
-constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + size_t(kStages) * kStageBytes + sizeof(SmemTail);
+template <bool PAIR>
+constexpr size_t smem_bytes() {
+    return 1024 /*alignment slack*/ + size_t(Plan<PAIR>::kStages) * Plan<PAIR>::kStageBytes + sizeof(SmemTail);
+}
 
 // ---------------------------------------------------------------- descriptors
 // Shared-memory matrix descriptor, 128-byte swizzle.  Bits: [0,14) address>>4, [16,30) leading
@@ -295,10 +305,15 @@ __device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const fl
 }
 
 // ---------------------------------------------------------------- the kernel
-template <int EPI, bool A_MN, bool B_MN>
+// PAIR = false: one CTA per 128 x 256 tile.  PAIR = true: a cluster of two CTAs per 256 x 256 tile
+// (tcgen05 cta_group::2): rank r loads rows [128 r, 128 r + 128) of the A tile and of the B tile,
+// rank 0 issues the MMAs for both, and each CTA drains its own 128 rows of the accumulator.
+template <int EPI, bool A_MN, bool B_MN, bool PAIR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
             const __grid_constant__ CUtensorMap tmB1, const GemmArgs p) {
+    constexpr int kStages = Plan<PAIR>::kStages;
+    constexpr int kStageBytes = Plan<PAIR>::kStageBytes;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;         // swizzle atoms need 1024-byte alignment
@@ -308,6 +323,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int num_tiles = p.num_m_tiles * p.num_n_tiles;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;             // rank in the CTA pair
+    const int first_tile = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+    const int tile_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
     volatile int* abort_flag = &tail->abort;
 
     if (threadIdx.x == 0) {
@@ -320,17 +338,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&tail->tmem_full[b]), 1);
-            mbar_init(smem_u32(&tail->tmem_empty[b]), kEpiThreads / 32);
+            mbar_init(smem_u32(&tail->tmem_empty[b]), (PAIR ? 2 : 1) * (kEpiThreads / 32));
         }
         tail->abort = 0;
         mbar_init_fence();
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols);
-        tmem_relinquish();
+        if constexpr (PAIR) { tmem_alloc_pair(smem_u32(&tail->tmem_base), kTmemCols); tmem_relinquish_pair(); }
+        else { tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols); tmem_relinquish(); }
     }
     tc_fence_before();
-    __syncthreads();
+    if constexpr (PAIR) cluster_sync_all(); else __syncthreads();   // barriers of both CTAs are ready
     tc_fence_after();
     const uint32_t tmem_base = tail->tmem_base;
 
@@ -339,37 +357,47 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            const CUtensorMap* tmB = (PAIR && rank != 0) ? &tmB1 : &tmB0;
+            for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
                 int m_tile, n_tile;
                 tile_coords(p, tile, m_tile, n_tile);
-                const int m0 = m_tile * kBlockM;
-                const int nb0 = n_tile * p.n_tile_cols;
+                const int m0 = m_tile * Plan<PAIR>::kTileM + static_cast<int>(rank) * kBlockM;
+                const int nb0 = n_tile * p.n_tile_cols + (PAIR ? static_cast<int>(rank) * p.b1_offset : 0);
                 const int nb1 = nb0 + p.b1_offset;
                 for (int kb = 0; kb < p.num_k_blocks; ++kb) {
                     if (!mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    const uint32_t bar = smem_u32(&tail->full[stage]);
                     const uint32_t dst = tiles_addr + stage * kStageBytes;
                     const int k0 = kb * kBlockK;
-                    mbar_expect_tx(bar, kStageBytes);
-                    if (A_MN) tma_load_2d(dst, &tmA, bar, m0, k0); else tma_load_2d(dst, &tmA, bar, k0, m0);
-                    if (B_MN) {
-                        tma_load_2d(dst + kBoxBytes, &tmB0, bar, nb0, k0);
-                        tma_load_2d(dst + 2 * kBoxBytes, &tmB1, bar, nb1, k0);
+                    if constexpr (PAIR) {
+                        // both CTAs' bytes are counted on rank 0's barrier, armed by rank 0 for both
+                        const uint32_t bar = mapa_shared(smem_u32(&tail->full[stage]), 0);
+                        if (rank == 0) mbar_expect_tx(smem_u32(&tail->full[stage]), 2 * kStageBytes);
+                        if (A_MN) tma_load_2d_pair(dst, &tmA, bar, m0, k0); else tma_load_2d_pair(dst, &tmA, bar, k0, m0);
+                        if (B_MN) tma_load_2d_pair(dst + kBoxBytes, tmB, bar, nb0, k0);
+                        else tma_load_2d_pair(dst + kBoxBytes, tmB, bar, k0, nb0);
                     } else {
-                        tma_load_2d(dst + kBoxBytes, &tmB0, bar, k0, nb0);
-                        tma_load_2d(dst + 2 * kBoxBytes, &tmB1, bar, k0, nb1);
+                        const uint32_t bar = smem_u32(&tail->full[stage]);
+                        mbar_expect_tx(bar, kStageBytes);
+                        if (A_MN) tma_load_2d(dst, &tmA, bar, m0, k0); else tma_load_2d(dst, &tmA, bar, k0, m0);
+                        if (B_MN) {
+                            tma_load_2d(dst + kBoxBytes, &tmB0, bar, nb0, k0);
+                            tma_load_2d(dst + 2 * kBoxBytes, &tmB1, bar, nb1, k0);
+                        } else {
+                            tma_load_2d(dst + kBoxBytes, &tmB0, bar, k0, nb0);
+                            tma_load_2d(dst + 2 * kBoxBytes, &tmB1, bar, k0, nb1);
+                        }
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (CTA pair: rank 0 only)
+        if (lane == 0 && rank == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             int it = 0;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+            for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step, ++it) {
                 const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(smem_u32(&tail->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, p.status)) break;
                 tc_fence_after();
@@ -383,12 +411,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                         const uint64_t da = smem_desc<A_MN>(a_addr + k * k_step_bytes<A_MN>());
                         const uint64_t db = smem_desc<B_MN>(b_addr + k * k_step_bytes<B_MN>());
-                        umma_f8(d_tmem, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                        if constexpr (PAIR) umma_f8_pair(d_tmem, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                        else umma_f8(d_tmem, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
                     }
-                    umma_commit(smem_u32(&tail->empty[stage]));      // frees the stage once these MMAs have read it
+                    // frees the stage (in both CTAs) once these MMAs have read it
+                    if constexpr (PAIR) umma_commit_pair(smem_u32(&tail->empty[stage]));
+                    else umma_commit(smem_u32(&tail->empty[stage]));
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) umma_commit(smem_u32(&tail->tmem_full[acc]));
+                if (ok) {
+                    if constexpr (PAIR) umma_commit_pair(smem_u32(&tail->tmem_full[acc]));
+                    else umma_commit(smem_u32(&tail->tmem_full[acc]));
+                }
             }
         }
     } else {
@@ -402,10 +436,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if constexpr (EPI == EPI_SWIGLU_BWD) sdz = *p.sdz;
         float run_max = 0.0f;
         int it = 0;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+        for (int tile = first_tile; tile < num_tiles; tile += tile_step, ++it) {
             int m_tile, n_tile;
             tile_coords(p, tile, m_tile, n_tile);
-            const int m = m_tile * kBlockM + row;
+            const int m = m_tile * Plan<PAIR>::kTileM + static_cast<int>(rank) * kBlockM + row;
             const int n0 = n_tile * p.n_tile_cols;
             const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
             if constexpr (EPI == EPI_SWIGLU_FWD) {
@@ -435,10 +469,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             } else {
                 run_max = fmaxf(run_max, epilogue_swiglu_bwd(p, tail->s_tile[acc], taddr, half, m, n0, dq0, sdz, gu_first));
             }
-            // accumulator drained: hand it back to the MMA warp
+            // accumulator drained: hand it back to the MMA warp (of rank 0)
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tail->tmem_empty[acc]));
+            if (lane == 0) {
+                if constexpr (PAIR) mbar_arrive_cluster(mapa_shared(smem_u32(&tail->tmem_empty[acc]), 0));
+                else mbar_arrive(smem_u32(&tail->tmem_empty[acc]));
+            }
             if constexpr (EPI == EPI_SWIGLU_FWD) {
                 epi_bar_sync();                        // all eight warps have merged into amax_tile
                 if (et < 128) {
@@ -463,10 +500,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
         __syncthreads();
     }
+    // neither CTA of a pair may leave while the other can still reach its shared or tensor memory
+    if constexpr (PAIR) cluster_sync_all();
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
+        if constexpr (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -488,24 +527,52 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-template <int EPI, bool A_MN, bool B_MN>
+template <int EPI, bool A_MN, bool B_MN, bool PAIR>
 int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorMap& tmB1, const GemmArgs& args,
-                int grid, cudaStream_t st) {
+                int64_t tiles, int sm_count, cudaStream_t st) {
+    constexpr size_t kSmem = smem_bytes<PAIR>();
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(kSmemBytes));
+    static int max_clusters = 0;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = kSmem;
+    cfg.stream = st;
+    if (PAIR) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(kSmem));
+        if (PAIR && attr_err == cudaSuccess) {
+            // how many CTA pairs the device can hold at once (one CTA per SM, pairs on neighbouring SMs)
+            cfg.gridDim = dim3(static_cast<unsigned>(sm_count) & ~1u);
+            attr_err = cudaOccupancyMaxActiveClusters(&max_clusters, gemm_kernel<EPI, A_MN, B_MN, PAIR>, &cfg);
+        }
     });
     FP8MLP_CUDA_CHECK(attr_err);
-    gemm_kernel<EPI, A_MN, B_MN><<<grid, kGemmThreads, kSmemBytes, st>>>(tmA, tmB0, tmB1, args);
-    FP8MLP_LAUNCH_CHECK();
+    int64_t grid;
+    if (PAIR) {
+        if (max_clusters < 1) { set_cuda_error_str("gemm launch", "no CTA pair fits on the device"); return FP8MLP_ERR_CUDA; }
+        grid = 2 * (tiles < max_clusters ? tiles : max_clusters);
+    } else {
+        grid = tiles < sm_count ? tiles : sm_count;
+    }
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    FP8MLP_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_kernel<EPI, A_MN, B_MN, PAIR>, tmA, tmB0, tmB1, args));
+    count_launch();
     return FP8MLP_OK;
 }
 
 }  // namespace
 
-size_t gemm_smem_bytes() { return kSmemBytes; }
+size_t gemm_smem_bytes() { return smem_bytes<true>() > smem_bytes<false>() ? smem_bytes<true>() : smem_bytes<false>(); }
 
 int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride) {
     EncodeTiledFn fn = encode_fn();
@@ -526,15 +593,18 @@ int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t ou
 
 int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUtensorMap& tmA, const CUtensorMap& tmB0,
                 const CUtensorMap& tmB1, GemmArgs args, int sm_count, cudaStream_t st) {
-    args.num_m_tiles = (args.M + kBlockM - 1) / kBlockM;
+    // a CTA pair works on 256 rows at a time; a problem of at most 128 rows runs on single CTAs
+    const bool pair = args.pair_mode == 1 || (args.pair_mode == 0 && args.M > kBlockM);
+    const int tile_m = pair ? 2 * kBlockM : kBlockM;
+    args.num_m_tiles = (args.M + tile_m - 1) / tile_m;
     args.num_n_tiles = (args.N + args.n_tile_cols - 1) / args.n_tile_cols;
     args.num_k_blocks = (args.K + kBlockK - 1) / kBlockK;
-    if (args.group_m <= 0) args.group_m = 16;
+    if (args.group_m <= 0) args.group_m = pair ? 8 : 16;
     // instruction descriptor: [4,6) D = fp32; [7,10) A format; [10,13) B format (0 = E4M3, 1 = E5M2);
-    // bit 15 / 16: A / B is MN-major; [17,23) N >> 3; [24,29) M >> 4
+    // bit 15 / 16: A / B is MN-major; [17,23) N >> 3; [24,29) M >> 4 (M counts both CTAs of a pair)
     args.idesc = (1u << 4) | (static_cast<uint32_t>(a_fmt) << 7) | (static_cast<uint32_t>(b_fmt) << 10) |
                  (static_cast<uint32_t>(a_mn) << 15) | (static_cast<uint32_t>(b_mn) << 16) |
-                 (static_cast<uint32_t>(kBlockN >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+                 (static_cast<uint32_t>(kBlockN >> 3) << 17) | (static_cast<uint32_t>(tile_m >> 4) << 24);
     // 32-byte stores need 32-byte aligned rows: the caller's pointers are only promised 16
     auto al32 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 31u) == 0; };
     switch (epi) {
@@ -545,10 +615,11 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     }
     const int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
     if (tiles == 0 || args.num_k_blocks == 0) return FP8MLP_OK;
-    const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);
 
-#define FP8MLP_DISPATCH(E, AM, BM) \
-    if (epi == E && a_mn == AM && b_mn == BM) return launch_inst<E, AM, BM>(tmA, tmB0, tmB1, args, grid, st);
+#define FP8MLP_DISPATCH(E, AM, BM)                                                                         \
+    if (epi == E && a_mn == AM && b_mn == BM)                                                              \
+        return pair ? launch_inst<E, AM, BM, true>(tmA, tmB0, tmB1, args, tiles, sm_count, st)             \
+                    : launch_inst<E, AM, BM, false>(tmA, tmB0, tmB1, args, tiles, sm_count, st);
     FP8MLP_DISPATCH(EPI_F32, false, false)
     FP8MLP_DISPATCH(EPI_F32, false, true)
     FP8MLP_DISPATCH(EPI_F32, true, false)

@@ -25,9 +25,7 @@ constexpr int kBlockM = 128;          // rows of D per tile (TMEM lanes)
 constexpr int kBlockN = 256;          // accumulator columns per tile
 constexpr int kBlockK = 128;          // contraction elements (= bytes) per pipeline stage
 constexpr int kUmmaK = 32;            // contraction elements per tcgen05.mma (32 bytes)
-constexpr int kStages = 4;
 constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 bytes x 128 rows
-constexpr int kStageBytes = 3 * kBoxBytes;   // A box + two B boxes
 constexpr int kGemmThreads = 320;
 constexpr int kTmemCols = 512;
 constexpr int kEpiThreads = 256;
@@ -38,6 +36,7 @@ struct GemmArgs {
     int n_tile_cols;        // n coordinates per tile: 256, or 128 when the two B boxes are gate and linear halves
     int b1_offset;          // n offset of the second B box: 128, or 0 in the gate/linear case
     int group_m;            // m-tiles per rasterisation band
+    int pair_mode;          // 0: CTA pairs when M > 128; 1: always CTA pairs; 2: always single CTAs
     uint32_t idesc;
     int* status;
 
