@@ -71,8 +71,8 @@ enum { /* fp8mlp_workspace: internal buffers, for inspection by tests */
 
 enum { /* phases of one step, for fp8mlp_profile_read (SMOOTH-mode kernel sequence) */
     FP8MLP_PH_QUANT_X = 0,    /* x -> E4M3 (+ amax)                                   */
-    FP8MLP_PH_QUANT_W12 = 1,  /* W2, W1 -> E4M3 [W2|W1] (+ amax)                      */
-    FP8MLP_PH_QUANT_W3 = 2,   /* 1/s, diag(1/s) W3 -> E4M3 (+ amax)                   */
+    FP8MLP_PH_QUANT_W12 = 1,  /* W2, W1 -> E4M3 [W2|W1] (+ amax); with given scales W3' too */
+    FP8MLP_PH_QUANT_W3 = 2,   /* diag(1/s) W3 -> E4M3 (+ amax), just-in-time scales only */
     FP8MLP_PH_GEMM1 = 3,      /* gate/up GEMM + SwiGLU / Smooth-SwiGLU epilogue       */
     FP8MLP_PH_GEMM2 = 4,      /* down projection                                      */
     FP8MLP_PH_QUANT_DY = 5,   /* dY -> E5M2 (+ amax)                                  */
@@ -117,8 +117,8 @@ FP8MLP_API int fp8mlp_profile_read(fp8mlp_ctx* ctx, double* ms, int64_t* count);
 /* Number of kernels this library has launched in this process so far (all contexts). */
 FP8MLP_API int64_t fp8mlp_launch_count(void);
 
-/* Per-tensor quantisation (Section 2: "scaling each tensor individually based on its specific
- * range of values"; Section 4.4 for row_mul).
+/* Per-tensor quantisation (Section 2: every tensor gets its own scale, chosen from its own
+ * range of values; Section 4.4 for row_mul).
  *   dst[r, c] = Q_fmt( (src[r, c] * row_mul[r]) * scale ),  r < rows, c < cols
  *   src       rows x cols, src_dtype FP8MLP_BF16 or FP8MLP_F32, contiguous.
  *   dst       FP8 codes, leading dimension ld_dst >= cols (bytes), ld_dst % 16 == 0.
@@ -175,7 +175,7 @@ FP8MLP_API int fp8mlp_backward(fp8mlp_ctx* ctx, int64_t T, const void* dy_bf16,
  * fail or fight that pool), or a serving loop that must not hit the device-wide synchronisation
  * and unpredictable latency a cudaMalloc / cudaFree can bring.  For them this entry point runs the
  * same forward as fp8mlp_forward (same kernels, forward only, nothing saved for backward) with the
- * internal buffers - the FP8 copies of x, [W2|W1], W3', the SwiGLU codes, 1/s and the status word -
+ * internal buffers - the FP8 copies of x, [W2|W1], W3', the SwiGLU codes and the status word -
  * placed in a fixed array that is part of the library image:
  *   FP8MLP_STATIC_SCRATCH_BYTES (4 MiB) of device memory, held by every GPU that loads the library
  *   until the process exits.  The problem fits when

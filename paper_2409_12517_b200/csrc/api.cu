@@ -24,10 +24,13 @@ void set_cuda_error_str(const char* what, const char* msg) {
 }
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
-// Sets up to 8 device floats to zero in one launch (amax accumulators).
-struct ZeroList { float* p[8]; };
+// Sets up to 8 device floats and one vector of floats to zero in one launch (amax accumulators).
+struct ZeroList { float* p[8]; float* vec; int64_t n; };
 __global__ void zero_floats_kernel(ZeroList z) {
-    if (threadIdx.x < 8 && z.p[threadIdx.x] != nullptr) *z.p[threadIdx.x] = 0.0f;
+    if (blockIdx.x == 0 && threadIdx.x < 8 && z.p[threadIdx.x] != nullptr) *z.p[threadIdx.x] = 0.0f;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < z.n;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x)
+        z.vec[i] = 0.0f;
 }
 
 }  // namespace fp8mlp
@@ -40,7 +43,6 @@ struct fp8mlp_ctx {
     int device, sm_count;
     uint8_t *xq, *w12q, *w3q, *hq, *dyq, *dzq;
     uint16_t* gu;
-    float* inv_s;     // [f] 1 / s_h: row multipliers of W3' = diag(s^-1) W3
     float* dummy;     // [8 + f] sinks for amax outputs the caller did not ask for
     int* status;      // bounded-wait status word
     int64_t saved_T;  // tokens of the last forward that saved activations, -1 if none
@@ -81,11 +83,14 @@ struct PhaseTimer {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int zero_floats(std::initializer_list<float*> ptrs, cudaStream_t st) {
+int zero_floats(std::initializer_list<float*> ptrs, cudaStream_t st, float* vec = nullptr, int64_t n_vec = 0) {
     ZeroList z{};
     int n = 0;
     for (float* p : ptrs) z.p[n++] = p;
-    zero_floats_kernel<<<1, 32, 0, st>>>(z);
+    z.vec = vec;
+    z.n = vec != nullptr ? n_vec : 0;
+    const int blocks = z.n > 256 ? static_cast<int>((z.n + 255) / 256 < 256 ? (z.n + 255) / 256 : 256) : 1;
+    zero_floats_kernel<<<blocks, 256, 0, st>>>(z);
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
 }
@@ -96,16 +101,20 @@ int zero_floats(std::initializer_list<float*> ptrs, cudaStream_t st) {
         if (rc__ != FP8MLP_OK) return rc__; \
     } while (0)
 
-// amax (optional) + cast of one tensor, in either scale mode.  amax must be non-null.
+// amax + cast of one tensor, in either scale mode.  amax must be non-null.
+// row_mul / row_div (both nullable): per-row multiplier, or per-row divisor (W3' = diag(s^-1) W3).
 int quantize_tensor(const void* src, int dtype, int64_t rows, int64_t cols, int fmt, int mode, float* scale,
-                    float* amax, const float* amax_other, const float* row_mul, uint8_t* dst, int64_t ld_dst,
-                    int sm_count, cudaStream_t st) {
+                    float* amax, const float* amax_other, const float* row_mul, const float* row_div, uint8_t* dst,
+                    int64_t ld_dst, int sm_count, cudaStream_t st) {
+    QuantTensor t{};
+    t.src = src; t.rows = rows; t.cols = cols; t.dst = dst; t.ld_dst = ld_dst; t.amax = amax;
+    t.row_mul = row_mul; t.row_div = row_div;
     if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
-        FP8MLP_TRY(run_quantize_pass(false, true, src, dtype, rows, cols, fmt, row_mul, nullptr, nullptr, 0, amax, sm_count, st));
+        FP8MLP_TRY(run_quantize_segments(false, true, dtype, fmt, &t, 1, nullptr, sm_count, st));
         FP8MLP_TRY(run_scale_from_amax(fmt, amax, amax_other, scale, st));
-        return run_quantize_pass(true, false, src, dtype, rows, cols, fmt, row_mul, scale, dst, ld_dst, nullptr, sm_count, st);
+        return run_quantize_segments(true, false, dtype, fmt, &t, 1, scale, sm_count, st);
     }
-    return run_quantize_pass(true, true, src, dtype, rows, cols, fmt, row_mul, scale, dst, ld_dst, amax, sm_count, st);
+    return run_quantize_segments(true, true, dtype, fmt, &t, 1, scale, sm_count, st);
 }
 
 GemmArgs base_args(fp8mlp_ctx* c, int M, int N, int K) {
@@ -127,14 +136,17 @@ int quantize_w12(fp8mlp_ctx* c, const float* W1, const float* W2, int mode, floa
     const int64_t d = c->d, f = c->f;
     const int sms = c->sm_count;
     if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
-        FP8MLP_TRY(run_quantize_pass(false, true, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, nullptr, nullptr, 0, a_w1, sms, st));
-        FP8MLP_TRY(run_quantize_pass(false, true, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, nullptr, nullptr, 0, a_w2, sms, st));
+        QuantTensor t[2] = {};
+        t[0].src = W2; t[0].rows = d; t[0].cols = f; t[0].dst = c->w12q; t[0].ld_dst = 2 * f; t[0].amax = a_w2;
+        t[1].src = W1; t[1].rows = d; t[1].cols = f; t[1].dst = c->w12q + f; t[1].ld_dst = 2 * f; t[1].amax = a_w1;
+        FP8MLP_TRY(run_quantize_segments(false, true, FP8MLP_F32, FP8MLP_E4M3, t, 2, nullptr, sms, st));
         FP8MLP_TRY(run_scale_from_amax(FP8MLP_E4M3, a_w1, a_w2, scale, st));
-        FP8MLP_TRY(run_quantize_pass(true, false, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, scale, c->w12q, 2 * f, nullptr, sms, st));
-        return run_quantize_pass(true, false, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, scale, c->w12q + f, 2 * f, nullptr, sms, st);
+        return run_quantize_segments(true, false, FP8MLP_F32, FP8MLP_E4M3, t, 2, scale, sms, st);
     }
-    FP8MLP_TRY(run_quantize_pass(true, true, W2, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, scale, c->w12q, 2 * f, a_w2, sms, st));
-    return run_quantize_pass(true, true, W1, FP8MLP_F32, d, f, FP8MLP_E4M3, nullptr, scale, c->w12q + f, 2 * f, a_w1, sms, st);
+    QuantTensor t[2] = {};
+    t[0].src = W2; t[0].rows = d; t[0].cols = f; t[0].dst = c->w12q; t[0].ld_dst = 2 * f; t[0].amax = a_w2;
+    t[1].src = W1; t[1].rows = d; t[1].cols = f; t[1].dst = c->w12q + f; t[1].ld_dst = 2 * f; t[1].amax = a_w1;
+    return run_quantize_segments(true, true, FP8MLP_F32, FP8MLP_E4M3, t, 2, scale, sms, st);
 }
 
 // G|U = Xq [W2q|W1q] with the SwiGLU / Smooth-SwiGLU epilogue
@@ -203,7 +215,6 @@ int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_
     void** slots[7] = {(void**)&c->xq, (void**)&c->w12q, (void**)&c->w3q, (void**)&c->hq,
                        (void**)&c->gu, (void**)&c->dyq, (void**)&c->dzq};
     for (int i = 0; i < 7 && e == cudaSuccess; ++i) e = cudaMalloc(slots[i], static_cast<size_t>(c->bytes[i]));
-    if (e == cudaSuccess) e = cudaMalloc((void**)&c->inv_s, sizeof(float) * f);
     if (e == cudaSuccess) e = cudaMalloc((void**)&c->dummy, sizeof(float) * (8 + f));
     if (e == cudaSuccess) e = cudaMalloc((void**)&c->status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int));
@@ -218,7 +229,7 @@ int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_
 
 int fp8mlp_destroy(fp8mlp_ctx* c) {
     if (c == nullptr) return FP8MLP_OK;
-    void* ptrs[] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq, c->inv_s, c->dummy, c->status};
+    void* ptrs[] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq, c->dummy, c->status};
     for (void* p : ptrs)
         if (p != nullptr) cudaFree(p);
     if (c->brackets != nullptr) {
@@ -291,7 +302,7 @@ int fp8mlp_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, 
     FP8MLP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     if (amax != nullptr) FP8MLP_TRY(zero_floats({amax}, st));
     if (scale_mode == FP8MLP_SCALE_FROM_CURRENT_AMAX)
-        return quantize_tensor(src, src_dtype, rows, cols, fp8_fmt, scale_mode, scale, amax, nullptr, row_mul, dst,
+        return quantize_tensor(src, src_dtype, rows, cols, fp8_fmt, scale_mode, scale, amax, nullptr, row_mul, nullptr, dst,
                                ld_dst, sms, st);
     return run_quantize_pass(true, amax != nullptr, src, src_dtype, rows, cols, fp8_fmt, row_mul, scale, dst, ld_dst,
                              amax, sms, st);
@@ -333,36 +344,42 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
 
     {
         PhaseTimer pt(c, FP8MLP_PH_MISC, st);
-        FP8MLP_TRY(zero_floats({a_x, a_w1, a_w2, a_w3}, st));
-        FP8MLP_CUDA_CHECK(cudaMemsetAsync(a_h, 0, sizeof(float) * f, st));
+        FP8MLP_TRY(zero_floats({a_x, a_w1, a_w2, a_w3}, st, a_h, f));
     }
     {   // x -> E4M3
         PhaseTimer pt(c, FP8MLP_PH_QUANT_X, st);
-        FP8MLP_TRY(quantize_tensor(x, FP8MLP_BF16, T, d, FP8MLP_E4M3, mode, sc->x, a_x, nullptr, nullptr, c->xq, d, c->sm_count, st));
+        FP8MLP_TRY(quantize_tensor(x, FP8MLP_BF16, T, d, FP8MLP_E4M3, mode, sc->x, a_x, nullptr, nullptr, nullptr, c->xq, d, c->sm_count, st));
     }
-    {   // [W2 | W1] -> E4M3 with one scale
+    if (mode == FP8MLP_SCALE_GIVEN) {
+        // every scale is known: [W2 | W1] (one scale) and W3' = diag(1/s) W3 in one pass over the masters;
+        // the reciprocal of s_i is taken inside the pass, row by row
         PhaseTimer pt(c, FP8MLP_PH_QUANT_W12, st);
-        FP8MLP_TRY(quantize_w12(c, W1, W2, mode, sc->w12, a_w1, a_w2, st));
-    }
-    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
+        QuantTensor t[3] = {};
+        t[0].src = W2; t[0].rows = d; t[0].cols = f; t[0].dst = c->w12q; t[0].ld_dst = 2 * f; t[0].amax = a_w2;
+        t[1].src = W1; t[1].rows = d; t[1].cols = f; t[1].dst = c->w12q + f; t[1].ld_dst = 2 * f; t[1].amax = a_w1;
+        t[2].src = W3; t[2].rows = f; t[2].cols = d; t[2].dst = c->w3q; t[2].ld_dst = d; t[2].amax = a_w3;
+        t[2].row_div = smooth ? sc->h : nullptr; t[2].scale = sc->w3;
+        FP8MLP_TRY(run_quantize_segments(true, true, FP8MLP_F32, FP8MLP_E4M3, t, 3, sc->w12, c->sm_count, st));
+    } else {
+        {   // [W2 | W1] -> E4M3 with one scale
+            PhaseTimer pt(c, FP8MLP_PH_QUANT_W12, st);
+            FP8MLP_TRY(quantize_w12(c, W1, W2, mode, sc->w12, a_w1, a_w2, st));
+        }
         // calibration pass: per-channel maxima of H, then s_i (or the per-tensor scale)
         if (T > 0) {
             PhaseTimer pt(c, FP8MLP_PH_GEMM1, st);
             FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/0, st));
         }
-        PhaseTimer pt(c, FP8MLP_PH_MISC, st);
-        UpdateScalesArgs u{};
-        u.amax_h = a_h; u.scale_h = sc->h; u.f = f; u.smooth = smooth ? 1 : 0;
-        FP8MLP_TRY(run_update_scales(u, c->sm_count, st));
-    }
-    {   // W3' = diag(1/s) W3 -> E4M3
-        PhaseTimer pt(c, FP8MLP_PH_QUANT_W3, st);
-        const float* row_mul = nullptr;
-        if (smooth) {
-            FP8MLP_TRY(run_reciprocal(sc->h, c->inv_s, f, st));
-            row_mul = c->inv_s;
+        {
+            PhaseTimer pt(c, FP8MLP_PH_MISC, st);
+            UpdateScalesArgs u{};
+            u.amax_h = a_h; u.scale_h = sc->h; u.f = f; u.smooth = smooth ? 1 : 0;
+            FP8MLP_TRY(run_update_scales(u, c->sm_count, st));
         }
-        FP8MLP_TRY(quantize_tensor(W3, FP8MLP_F32, f, d, FP8MLP_E4M3, mode, sc->w3, a_w3, nullptr, row_mul, c->w3q, d, c->sm_count, st));
+        // W3' = diag(1/s) W3 -> E4M3
+        PhaseTimer pt(c, FP8MLP_PH_QUANT_W3, st);
+        FP8MLP_TRY(quantize_tensor(W3, FP8MLP_F32, f, d, FP8MLP_E4M3, mode, sc->w3, a_w3, nullptr, nullptr,
+                                   smooth ? sc->h : nullptr, c->w3q, d, c->sm_count, st));
     }
     if (T == 0) { c->saved_T = (c->flags & FP8MLP_SAVE_FOR_BWD) ? 0 : -1; return FP8MLP_OK; }
     {
@@ -413,7 +430,7 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
 
     {   // dY -> E5M2
         PhaseTimer pt(c, FP8MLP_PH_QUANT_DY, st);
-        FP8MLP_TRY(quantize_tensor(dy, FP8MLP_BF16, T, d, FP8MLP_E5M2, mode, sc->dy, a_dy, nullptr, nullptr, c->dyq, d, c->sm_count, st));
+        FP8MLP_TRY(quantize_tensor(dy, FP8MLP_BF16, T, d, FP8MLP_E5M2, mode, sc->dy, a_dy, nullptr, nullptr, nullptr, c->dyq, d, c->sm_count, st));
     }
 
     // dH~ = dYq W3q^T with the SwiGLU-backward epilogue -> dZq = [dG | dU]
@@ -520,7 +537,6 @@ int fp8mlp_forward_static(int64_t T, int64_t d, int64_t f, uint32_t flags, const
     auto carve = [&](int64_t bytes) { unsigned char* p = base + off; off += round_up_256(bytes); return p; };
     c.status = reinterpret_cast<int*>(carve(256));
     c.dummy = reinterpret_cast<float*>(carve(sizeof(float) * (8 + f)));
-    c.inv_s = reinterpret_cast<float*>(carve(sizeof(float) * f));
     c.xq = carve(T * d);
     c.w12q = carve(2 * d * f);
     c.w3q = carve(f * d);

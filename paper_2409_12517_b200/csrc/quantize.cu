@@ -50,68 +50,111 @@ __device__ __forceinline__ void block_atomic_max(float v, float* out) {
     }
 }
 
-// Loads 16 consecutive source elements as fp32.
+// A unit is 32 bytes of source: 8 fp32 or 16 bf16 elements.  Lane l of a warp takes unit l of the
+// warp's 1 KiB, so every load instruction of a warp covers whole 128-byte lines.
+template <typename SRC> struct Unit;
+template <> struct Unit<float> { static constexpr int kElems = 8; };
+template <> struct Unit<uint16_t> { static constexpr int kElems = 16; };
+
 template <typename SRC>
-__device__ __forceinline__ void load16(const SRC* p, float (&v)[16]);
-
-template <>
-__device__ __forceinline__ void load16<float>(const float* p, float (&v)[16]) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        uint4 q = ld_global_nc_v4(p + 4 * i);
-        v[4 * i + 0] = __uint_as_float(q.x);
-        v[4 * i + 1] = __uint_as_float(q.y);
-        v[4 * i + 2] = __uint_as_float(q.z);
-        v[4 * i + 3] = __uint_as_float(q.w);
-    }
-}
-template <>
-__device__ __forceinline__ void load16<uint16_t>(const uint16_t* p, float (&v)[16]) {   // bf16 bits
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        uint4 q = ld_global_nc_v4(p + 8 * i);
-        v[8 * i + 0] = bf16_lo(q.x); v[8 * i + 1] = bf16_hi(q.x);
-        v[8 * i + 2] = bf16_lo(q.y); v[8 * i + 3] = bf16_hi(q.y);
-        v[8 * i + 4] = bf16_lo(q.z); v[8 * i + 5] = bf16_hi(q.z);
-        v[8 * i + 6] = bf16_lo(q.w); v[8 * i + 7] = bf16_hi(q.w);
+__device__ __forceinline__ void load_unit(const SRC* p, bool wide, uint32_t (&w)[8]) {
+    if (wide) {
+        ld_global_nc_v8(p, w);
+    } else {   // the base is only 16-byte aligned
+        const uint4 lo = ld_global_nc_v4(p), hi = ld_global_nc_v4(reinterpret_cast<const uint8_t*>(p) + 16);
+        w[0] = lo.x; w[1] = lo.y; w[2] = lo.z; w[3] = lo.w; w[4] = hi.x; w[5] = hi.y; w[6] = hi.z; w[7] = hi.w;
     }
 }
 
-// One pass over src in chunks of 16 elements.  CAST: write FP8 codes; AMAX: reduce max |v|.
-// chunks_per_row = cols / 16.  row_mul (nullable) multiplies row r before anything else.
+template <typename SRC>
+__device__ __forceinline__ void unpack_unit(const uint32_t (&w)[8], float (&v)[Unit<SRC>::kElems]);
+template <>
+__device__ __forceinline__ void unpack_unit<float>(const uint32_t (&w)[8], float (&v)[8]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(w[i]);
+}
+template <>
+__device__ __forceinline__ void unpack_unit<uint16_t>(const uint32_t (&w)[8], float (&v)[16]) {   // bf16 bits
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { v[2 * i] = bf16_lo(w[i]); v[2 * i + 1] = bf16_hi(w[i]); }
+}
+
+// One pass over up to kMaxQuantSegs tensors ("segments": e.g. W2 and W1, which become the two column
+// halves of one FP8 operand, and W3').  Blocks are dealt to the segments round-robin;
+// kUnroll 32-byte loads in flight per thread.
+// CAST: write FP8 codes; AMAX: reduce max |v| into the segment's amax.
+constexpr int kUnroll = 4;
+constexpr int kBlocksPerSm = 3;
+
 template <typename SRC, int FMT, bool CAST, bool AMAX>
-__global__ void __launch_bounds__(kThreads)
-quantize_kernel(const SRC* __restrict__ src, int64_t n_chunks, int64_t chunks_per_row,
-                const float* __restrict__ row_mul, const float* __restrict__ scale_ptr,
-                uint8_t* __restrict__ dst, int64_t ld_dst, float* __restrict__ amax_out) {
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm)
+quantize_kernel(const QuantLaunch q) {
+    constexpr int E = Unit<SRC>::kElems;
+    const int seg_id = blockIdx.x % q.nseg;
+    const QuantSeg& sg = q.seg[seg_id];
+    const SRC* __restrict__ src = static_cast<const SRC*>(sg.src);
     float scale = 1.0f;
-    if constexpr (CAST) scale = *scale_ptr;
+    if constexpr (CAST) scale = *sg.scale;
     float local_max = 0.0f;
-    const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
-    for (int64_t q = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; q < n_chunks; q += stride) {
-        float v[16];
-        load16<SRC>(src + q * 16, v);
-        const int64_t r = q / chunks_per_row;
-        if (row_mul != nullptr) {
-            const float m = row_mul[r];
+    // every block of a segment owns an equal, contiguous range of units: all blocks end together
+    const uint32_t begin = (blockIdx.x / q.nseg) * q.units_per_block;
+    const uint32_t end = min(begin + q.units_per_block, sg.n_units);
+    const bool has_row = sg.row_mul != nullptr || sg.row_div != nullptr;
+    const bool flat = !has_row && sg.ld_dst == static_cast<int64_t>(sg.units_per_row) * E;
+    // (row, column unit) of this thread's next unit, advanced by kThreads units at a time: one
+    // division per thread instead of one per unit
+    const uint32_t upr = sg.units_per_row;
+    uint32_t next_row = (begin + threadIdx.x) / upr;
+    uint32_t next_col = (begin + threadIdx.x) - next_row * upr;
+    for (uint32_t u0 = begin + threadIdx.x; u0 < end; u0 += kThreads * kUnroll) {
+        uint32_t w[kUnroll][8];
+        uint32_t row[kUnroll], col[kUnroll];
+        float mul[kUnroll];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(v[i], m);
+        for (int k = 0; k < kUnroll; ++k) {
+            const uint32_t u = u0 + k * kThreads;
+            row[k] = next_row;
+            col[k] = next_col;
+            if (u < end) {
+                load_unit<SRC>(src + static_cast<int64_t>(u) * E, q.wide != 0, w[k]);
+                if (has_row) mul[k] = sg.row_div != nullptr ? sg.row_div[next_row] : sg.row_mul[next_row];
+            }
+            if (!flat) {
+                next_col += kThreads;
+                while (next_col >= upr) { next_col -= upr; ++next_row; }
+            }
         }
-        if constexpr (AMAX) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) local_max = fmaxf(local_max, fabsf(v[i]));
-        }
-        if constexpr (CAST) {
-            uint32_t w[4];
+        for (int k = 0; k < kUnroll; ++k) {
+            const uint32_t u = u0 + k * kThreads;
+            if (u >= end) break;
+            float v[E];
+            unpack_unit<SRC>(w[k], v);
+            int64_t out = static_cast<int64_t>(u) * E;
+            if (!flat) {
+                out = static_cast<int64_t>(row[k]) * sg.ld_dst + static_cast<int64_t>(col[k]) * E;
+                if (has_row) {
+                    const float m = sg.row_div != nullptr ? __fdiv_rn(1.0f, mul[k]) : mul[k];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                w[i] = cvt_fp8x4<FMT>(__fmul_rn(v[4 * i], scale), __fmul_rn(v[4 * i + 1], scale),
-                                      __fmul_rn(v[4 * i + 2], scale), __fmul_rn(v[4 * i + 3], scale));
-            const int64_t c = (q - r * chunks_per_row) * 16;
-            st_global_v4(dst + r * ld_dst + c, w[0], w[1], w[2], w[3]);
+                    for (int i = 0; i < E; ++i) v[i] = __fmul_rn(v[i], m);
+                }
+            }
+            if constexpr (AMAX) {
+#pragma unroll
+                for (int i = 0; i < E; ++i) local_max = fmaxf(local_max, fabsf(v[i]));
+            }
+            if constexpr (CAST) {
+                uint32_t c[E / 4];
+#pragma unroll
+                for (int i = 0; i < E / 4; ++i)
+                    c[i] = cvt_fp8x4<FMT>(__fmul_rn(v[4 * i], scale), __fmul_rn(v[4 * i + 1], scale),
+                                          __fmul_rn(v[4 * i + 2], scale), __fmul_rn(v[4 * i + 3], scale));
+                if constexpr (E == 16) st_global_v4(sg.dst + out, c[0], c[1], c[2], c[3]);
+                else st_global_v2(sg.dst + out, c[0], c[1]);
+            }
         }
     }
-    if constexpr (AMAX) block_atomic_max(local_max, amax_out);
+    if constexpr (AMAX) block_atomic_max(local_max, sg.amax);
 }
 
 // scale = fmt_max / max(amax_a, amax_b)   (amax_b nullable)
@@ -158,53 +201,82 @@ __global__ void __launch_bounds__(kThreads) update_scales_kernel(UpdateScalesArg
     }
 }
 
-// out[i] = 1 / s[i]   (row multipliers for W3' = diag(s^-1) W3)
-__global__ void __launch_bounds__(kThreads) reciprocal_kernel(const float* __restrict__ s, float* __restrict__ out, int64_t n) {
-    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < n;
-         i += static_cast<int64_t>(gridDim.x) * kThreads)
-        out[i] = __fdiv_rn(1.0f, s[i]);
-}
-
-int grid_for(int64_t n_chunks, int sm_count) {
-    // enough blocks to keep every SM's load queues full; a multiple of the SM count
-    int64_t want = (n_chunks + kThreads - 1) / kThreads;
-    int64_t cap = static_cast<int64_t>(sm_count) * 8;
-    if (want < 1) want = 1;
-    return static_cast<int>(want < cap ? want : cap);
-}
-
 template <typename SRC, int FMT>
-int launch_pass(bool cast, bool amax, const SRC* src, int64_t n_chunks, int64_t cpr, const float* row_mul,
-                const float* scale, uint8_t* dst, int64_t ld_dst, float* amax_out, int sm_count, cudaStream_t st) {
-    const int grid = grid_for(n_chunks, sm_count);
-    if (cast && amax)
-        quantize_kernel<SRC, FMT, true, true><<<grid, kThreads, 0, st>>>(src, n_chunks, cpr, row_mul, scale, dst, ld_dst, amax_out);
-    else if (cast)
-        quantize_kernel<SRC, FMT, true, false><<<grid, kThreads, 0, st>>>(src, n_chunks, cpr, row_mul, scale, dst, ld_dst, amax_out);
-    else
-        quantize_kernel<SRC, FMT, false, true><<<grid, kThreads, 0, st>>>(src, n_chunks, cpr, row_mul, scale, dst, ld_dst, amax_out);
+int launch_pass(bool cast, bool amax, const QuantLaunch& q, int grid, cudaStream_t st) {
+    if (cast && amax) quantize_kernel<SRC, FMT, true, true><<<grid, kThreads, 0, st>>>(q);
+    else if (cast) quantize_kernel<SRC, FMT, true, false><<<grid, kThreads, 0, st>>>(q);
+    else quantize_kernel<SRC, FMT, false, true><<<grid, kThreads, 0, st>>>(q);
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
 }
 
 }  // namespace
 
+int run_quantize_segments(bool cast, bool amax, int src_dtype, int fmt, const QuantTensor* t, int nseg,
+                          const float* scale, int sm_count, cudaStream_t st) {
+    if (nseg < 1 || nseg > kMaxQuantSegs) return FP8MLP_ERR_ARG;
+    const int elems = src_dtype == FP8MLP_F32 ? 8 : 16;
+    // unit indices are 32-bit: tensors beyond 2^31 units are cut into row blocks
+    const int64_t kMaxUnits = int64_t(1) << 31;
+    int64_t worst = 0;
+    for (int i = 0; i < nseg; ++i) {
+        const int64_t units = t[i].rows * (t[i].cols / elems);
+        if (units > worst) worst = units;
+    }
+    if (worst == 0) return FP8MLP_OK;
+    if (worst > kMaxUnits) {
+        for (int i = 0; i < nseg; ++i) {
+            const int64_t upr = t[i].cols / elems;
+            if (upr == 0 || t[i].rows == 0) continue;
+            const int64_t rows_per = kMaxUnits / upr > 0 ? kMaxUnits / upr : 1;
+            for (int64_t r0 = 0; r0 < t[i].rows; r0 += rows_per) {
+                QuantTensor part = t[i];
+                part.rows = t[i].rows - r0 < rows_per ? t[i].rows - r0 : rows_per;
+                part.src = static_cast<const uint8_t*>(t[i].src) + r0 * t[i].cols * (src_dtype == FP8MLP_F32 ? 4 : 2);
+                if (part.dst != nullptr) part.dst += r0 * t[i].ld_dst;
+                if (part.row_mul != nullptr) part.row_mul += r0;
+                if (part.row_div != nullptr) part.row_div += r0;
+                int rc = run_quantize_segments(cast, amax, src_dtype, fmt, &part, 1, scale, sm_count, st);
+                if (rc != FP8MLP_OK) return rc;
+            }
+        }
+        return FP8MLP_OK;
+    }
+    QuantLaunch q{};
+    q.nseg = nseg;
+    q.scale = scale;
+    q.wide = 1;
+    for (int i = 0; i < nseg; ++i) {
+        QuantSeg& sg = q.seg[i];
+        sg.src = t[i].src; sg.dst = t[i].dst; sg.amax = t[i].amax;
+        sg.row_mul = t[i].row_mul; sg.row_div = t[i].row_div;
+        sg.scale = t[i].scale != nullptr ? t[i].scale : scale;
+        sg.units_per_row = static_cast<uint32_t>(t[i].cols / elems);
+        sg.n_units = static_cast<uint32_t>(t[i].rows * (t[i].cols / elems));
+        sg.ld_dst = t[i].ld_dst;
+        if (reinterpret_cast<uintptr_t>(t[i].src) & 31u) q.wide = 0;
+    }
+    // every resident block slot of the device gets one block (fewer for small tensors), the same number
+    // for every segment, and each block an equal share of its segment, rounded up to whole warps
+    int64_t per_seg = static_cast<int64_t>(sm_count) * kBlocksPerSm / nseg;
+    const int64_t enough = (worst + int64_t(kThreads) * kUnroll - 1) / (int64_t(kThreads) * kUnroll);
+    if (per_seg > enough) per_seg = enough;
+    if (per_seg < 1) per_seg = 1;
+    q.units_per_block = static_cast<uint32_t>(((worst + per_seg - 1) / per_seg + 31) / 32 * 32);
+    const int grid = static_cast<int>(per_seg) * nseg;
+    if (src_dtype == FP8MLP_F32)
+        return fmt == FP8MLP_E4M3 ? launch_pass<float, FP8MLP_E4M3>(cast, amax, q, grid, st)
+                                  : launch_pass<float, FP8MLP_E5M2>(cast, amax, q, grid, st);
+    return fmt == FP8MLP_E4M3 ? launch_pass<uint16_t, FP8MLP_E4M3>(cast, amax, q, grid, st)
+                              : launch_pass<uint16_t, FP8MLP_E5M2>(cast, amax, q, grid, st);
+}
+
 int run_quantize_pass(bool cast, bool amax, const void* src, int src_dtype, int64_t rows, int64_t cols, int fmt,
                       const float* row_mul, const float* scale, uint8_t* dst, int64_t ld_dst, float* amax_out,
                       int sm_count, cudaStream_t st) {
-    const int64_t cpr = cols / 16;
-    const int64_t n_chunks = rows * cpr;
-    if (n_chunks == 0) return FP8MLP_OK;
-    if (src_dtype == FP8MLP_F32) {
-        const float* s = static_cast<const float*>(src);
-        return fmt == FP8MLP_E4M3
-                   ? launch_pass<float, FP8MLP_E4M3>(cast, amax, s, n_chunks, cpr, row_mul, scale, dst, ld_dst, amax_out, sm_count, st)
-                   : launch_pass<float, FP8MLP_E5M2>(cast, amax, s, n_chunks, cpr, row_mul, scale, dst, ld_dst, amax_out, sm_count, st);
-    }
-    const uint16_t* s = static_cast<const uint16_t*>(src);
-    return fmt == FP8MLP_E4M3
-               ? launch_pass<uint16_t, FP8MLP_E4M3>(cast, amax, s, n_chunks, cpr, row_mul, scale, dst, ld_dst, amax_out, sm_count, st)
-               : launch_pass<uint16_t, FP8MLP_E5M2>(cast, amax, s, n_chunks, cpr, row_mul, scale, dst, ld_dst, amax_out, sm_count, st);
+    QuantTensor t{};
+    t.src = src; t.rows = rows; t.cols = cols; t.dst = dst; t.ld_dst = ld_dst; t.amax = amax_out; t.row_mul = row_mul;
+    return run_quantize_segments(cast, amax, src_dtype, fmt, &t, 1, scale, sm_count, st);
 }
 
 int run_scale_from_amax(int fmt, const float* amax_a, const float* amax_b, float* scale, cudaStream_t st) {
@@ -218,15 +290,6 @@ int run_update_scales(const UpdateScalesArgs& a, int sm_count, cudaStream_t st) 
     if (blocks < 1) blocks = 1;
     if (blocks > sm_count) blocks = sm_count;
     update_scales_kernel<<<static_cast<int>(blocks), kThreads, 0, st>>>(a);
-    FP8MLP_LAUNCH_CHECK();
-    return FP8MLP_OK;
-}
-
-int run_reciprocal(const float* s, float* out, int64_t n, cudaStream_t st) {
-    if (n == 0) return FP8MLP_OK;
-    int64_t blocks = (n + kThreads - 1) / kThreads;
-    if (blocks > 1024) blocks = 1024;
-    reciprocal_kernel<<<static_cast<int>(blocks), kThreads, 0, st>>>(s, out, n);
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
 }

@@ -5,6 +5,28 @@
 
 namespace fp8mlp {
 
+// Tensors of one source dtype and FP8 format quantised together in one launch (e.g. W2 and W1, the
+// two column halves of one FP8 operand, and W3'), each with its own amax and scale pointer.
+constexpr int kMaxQuantSegs = 3;
+struct QuantTensor {
+    const void* src;        // rows x cols, contiguous, 16-byte aligned
+    int64_t rows, cols;     // cols % 16 == 0
+    uint8_t* dst;           // codes, leading dimension ld_dst (cast passes)
+    int64_t ld_dst;
+    float* amax;            // raised atomically to max |src * multiplier| (amax passes; zeroed by the caller)
+    const float* row_mul;   // nullable: row r is multiplied by row_mul[r] first
+    const float* row_div;   // nullable: row r is multiplied by 1 / row_div[r] first (W3' = diag(s^-1) W3)
+    const float* scale;     // nullable: overrides the launch's scale for this tensor
+};
+// what the kernel sees
+struct QuantSeg {
+    const void* src; uint8_t* dst; float* amax; const float* row_mul; const float* row_div; const float* scale;
+    int64_t ld_dst; uint32_t units_per_row, n_units;
+};
+struct QuantLaunch { QuantSeg seg[kMaxQuantSegs]; int nseg; int wide; uint32_t units_per_block; const float* scale; };
+int run_quantize_segments(bool cast, bool amax, int src_dtype, int fmt, const QuantTensor* t, int nseg,
+                          const float* scale, int sm_count, cudaStream_t st);
+
 // One streaming pass over a rows x cols tensor (cols % 16 == 0).
 //   cast: write FP8 codes dst[r*ld_dst + c] = Q((src*row_mul[r]) * *scale)
 //   amax: atomically raise *amax_out to max |src*row_mul| (the caller zeroes it first)
@@ -23,7 +45,5 @@ struct UpdateScalesArgs {
 };
 int run_update_scales(const UpdateScalesArgs& a, int sm_count, cudaStream_t st);
 
-// out[i] = 1 / s[i]
-int run_reciprocal(const float* s, float* out, int64_t n, cudaStream_t st);
 
 }  // namespace fp8mlp
