@@ -217,8 +217,11 @@ __device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
+// Arrival on a barrier that may sit in the partner CTA.  What it hands over is tensor memory
+// (ordered by tcgen05.fence), not global data, so the default CTA-scope release is enough and the
+// warp does not wait for its global stores to be acknowledged.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // 2-D tile load into this CTA's shared memory whose bytes are counted on a barrier that may sit in
 // the partner CTA (`bar_cluster` is a shared::cluster address).  No multicast.
