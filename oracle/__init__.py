@@ -16,6 +16,8 @@ import numpy as np
 _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "fp8mlp_oracle.c"
 _LIB = _HERE / "liboracle.so"
+_ADAM_SRC = _HERE / "fp8adam_oracle.c"
+_ADAM_LIB = _HERE / "liboracle_adam.so"
 
 E4M3, E5M2 = 0, 1
 FLAG_SMOOTH, FLAG_Q_IDENTITY, FLAG_NO_BF16 = 1, 2, 4
@@ -31,6 +33,11 @@ def build(force: bool = False) -> Path:
         subprocess.check_call(["gcc", "-O2", "-fopenmp", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC",
                                "-o", str(tmp), str(_SRC), "-lm"])
         os.replace(tmp, _LIB)
+    if force or not _ADAM_LIB.exists() or _ADAM_LIB.stat().st_mtime < _ADAM_SRC.stat().st_mtime:
+        tmp = _ADAM_LIB.with_suffix(f".so.tmp{os.getpid()}")
+        subprocess.check_call(["gcc", "-O2", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC",
+                               "-o", str(tmp), str(_ADAM_SRC), "-lm"])
+        os.replace(tmp, _ADAM_LIB)
     return _LIB
 
 
@@ -252,3 +259,53 @@ def mlp_f64_backward(x, W1, W2, W3, dY):
     lib().orc_mlp_f64_backward(C.c_int64(T), C.c_int64(d), C.c_int64(f), _p(x), _p(W1), _p(W2), _p(W3), _p(dY),
                                _p(dX), _p(dW1), _p(dW2), _p(dW3))
     return dX, dW1, dW2, dW3
+
+
+# ---------------------------------------------------------------- Adam with FP8 moments (fp8adam_oracle.c)
+ADAM_Q_IDENTITY, ADAM_M_AS_E5M2, ADAM_V_AS_E4M3 = 1, 2, 4
+_adam = None
+
+
+def _adam_lib():
+    global _adam
+    if _adam is None:
+        build()
+        _adam = C.CDLL(str(_ADAM_LIB))
+        _adam.adam_decode.restype = C.c_float
+        _adam.adam_decode.argtypes = [C.c_int, C.c_uint8]
+        _adam.adam_encode.restype = C.c_uint8
+        _adam.adam_encode.argtypes = [C.c_int, C.c_float]
+        _adam.adam_bias_correction.restype = C.c_float
+        _adam.adam_bias_correction.argtypes = [C.c_float, C.c_int64]
+        _adam.adam_step.restype = None
+    return _adam
+
+
+def adam_encode(second_moment: bool, v: float) -> int:
+    return int(_adam_lib().adam_encode(int(second_moment), np.float32(v)))
+
+
+def adam_decode(second_moment: bool, code: int) -> float:
+    return float(_adam_lib().adam_decode(int(second_moment), code))
+
+
+def adam_bias_correction(beta: float, step: int) -> float:
+    return float(_adam_lib().adam_bias_correction(np.float32(beta), step))
+
+
+def adam_step(w, g, mq, vq, *, lr, beta1, beta2, eps, weight_decay, step, sm_in=1.0, sv_in=1.0, sm_out=1.0,
+              sv_out=1.0, m32=None, v32=None, flags=0):
+    """One Adam step in place (w fp32; mq, vq uint8 codes, or m32, v32 fp32 with the quantisation off).
+    Returns (amax_m, amax_v) of the new fp32 moments."""
+    assert w.dtype == np.float32 and g.dtype == np.float32 and w.flags.c_contiguous and g.flags.c_contiguous
+    if m32 is not None:
+        flags |= ADAM_Q_IDENTITY
+        assert m32.dtype == np.float32 and v32.dtype == np.float32
+    else:
+        assert mq.dtype == np.uint8 and vq.dtype == np.uint8
+    am, av = C.c_float(0), C.c_float(0)
+    _adam_lib().adam_step(C.c_int64(w.size), C.c_uint(flags), _p(w), _p(g), _p(mq), _p(vq), _p(m32), _p(v32),
+                          C.c_float(lr), C.c_float(beta1), C.c_float(beta2), C.c_float(eps), C.c_float(weight_decay),
+                          C.c_int64(step), C.c_float(sm_in), C.c_float(sv_in), C.c_float(sm_out), C.c_float(sv_out),
+                          C.byref(am), C.byref(av))
+    return float(am.value), float(av.value)
