@@ -168,6 +168,42 @@ FP8MLP_API int fp8mlp_backward(fp8mlp_ctx* ctx, int64_t T, const void* dy_bf16,
                     int scale_mode, fp8mlp_scales* scales, fp8mlp_amax* amax,
                     void* dx_bf16, float* dW1, float* dW2, float* dW3, void* stream);
 
+/* Adam step with both moments stored in FP8 (Section 5: first moment E4M3, second moment E5M2 -
+ * the update divides by the square root of the second moment, so its smallest values matter and it
+ * needs the wider exponent range).  The step after fp8mlp_backward: it consumes dW1, dW2, dW3.
+ * The update is the textbook one (bias-corrected Adam, decoupled weight decay); per parameter i,
+ * in fp32, one rounding per operation in this order:
+ *   m_prev = dec_e4m3(m[i]) * (1 / *scale_m_in);     v_prev = dec_e5m2(v[i]) * (1 / *scale_v_in)
+ *   mi = beta1 * m_prev + (1 - beta1) * g[i];        vi = beta2 * v_prev + (1 - beta2) * (g[i] * g[i])
+ *   upd = (mi * c1) / (sqrt(vi * c2) + eps) [+ weight_decay * w[i]],   c = 1 / (1 - beta^step) (fp64, rounded once)
+ *   w[i] = w[i] - lr * upd
+ *   m[i] = Q_e4m3(mi * *scale_m_out);                v[i] = Q_e5m2(vi * *scale_v_out)
+ *   *amax_m = max |mi|;  *amax_v = max vi            (of the fp32 moments, for the next step's scales)
+ * Scaling is per tensor and delayed, like the rest of the recipe: the caller keeps, per tensor, the
+ * scale the stored codes were written with (`in`) and chooses the scale to write with (`out`), e.g.
+ * with fp8mlp_scale_from_amax on the maxima of the previous step; `in` and `out` may be the same
+ * buffer.  A zero state is codes 0 with scales 1.
+ * Up to 8 tensors per call (one launch); n % 16 == 0; w, g fp32 and m, v FP8 codes, device pointers,
+ * 16-byte aligned, updated in place; scales and maxima device floats.  step >= 1. */
+typedef struct {
+    float* w;                  /* [n] master weights, updated in place        */
+    const float* g;            /* [n] gradients                                */
+    uint8_t* m;                /* [n] first moment, E4M3 codes, in place       */
+    uint8_t* v;                /* [n] second moment, E5M2 codes, in place      */
+    int64_t n;
+    const float* scale_m_in;   /* scales the stored codes were written with    */
+    const float* scale_v_in;
+    const float* scale_m_out;  /* scales the new codes are written with        */
+    const float* scale_v_out;
+    float* amax_m;             /* out: max |m|, max v of this step's moments   */
+    float* amax_v;
+} fp8mlp_adam_tensor;
+FP8MLP_API int fp8mlp_adam_step(const fp8mlp_adam_tensor* tensors, int count, float lr, float beta1, float beta2,
+                                float eps, float weight_decay, int64_t step, void* stream);
+/* *scale = fmt_max / *amax (Section 2, per-tensor scaling; 1 if *amax is zero or not finite).
+ * fp8_fmt FP8MLP_E4M3 or FP8MLP_E5M2; both pointers device floats. */
+FP8MLP_API int fp8mlp_scale_from_amax(const float* amax, int fp8_fmt, float* scale, void* stream);
+
 /* Forward without any allocation (the paper has no counterpart; this is a deployment aid).
  *
  * Some callers cannot create a context because they cannot allocate device memory at all: a plug-in

@@ -27,7 +27,7 @@ EXPORTS = [
     "fp8mlp_create", "fp8mlp_destroy", "fp8mlp_strerror", "fp8mlp_last_cuda_error", "fp8mlp_status",
     "fp8mlp_workspace", "fp8mlp_launch_count", "fp8mlp_quantize", "fp8mlp_update_scales",
     "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8", "fp8mlp_profile_enable", "fp8mlp_profile_read",
-    "fp8mlp_forward_static",
+    "fp8mlp_forward_static", "fp8mlp_adam_step", "fp8mlp_scale_from_amax",
 ]
 PHASES = ["quant_x", "quant_w12", "quant_w3", "gemm1_swiglu", "gemm2_down", "quant_dy", "dgrad2_swiglu_bwd",
           "wgrad3", "dgrad1", "wgrad12", "misc"]
@@ -47,6 +47,12 @@ class _Scales(C.Structure):
 
 class _Amax(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("x", "w1", "w2", "w3", "dy", "dz", "h")]
+
+
+class _AdamTensor(C.Structure):
+    _fields_ = [("w", C.c_void_p), ("g", C.c_void_p), ("m", C.c_void_p), ("v", C.c_void_p), ("n", C.c_int64),
+                ("scale_m_in", C.c_void_p), ("scale_v_in", C.c_void_p), ("scale_m_out", C.c_void_p),
+                ("scale_v_out", C.c_void_p), ("amax_m", C.c_void_p), ("amax_v", C.c_void_p)]
 
 
 _lib = None
@@ -80,6 +86,9 @@ def lib():
         L.fp8mlp_forward_static.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_uint32, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_int, C.POINTER(_Scales), C.POINTER(_Amax),
                                             C.c_void_p, C.c_void_p]
+        L.fp8mlp_adam_step.argtypes = [C.POINTER(_AdamTensor), C.c_int, C.c_float, C.c_float, C.c_float, C.c_float,
+                                       C.c_float, C.c_int64, C.c_void_p]
+        L.fp8mlp_scale_from_amax.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         L.fp8mlp_profile_enable.argtypes = [C.c_void_p, C.c_int]
         L.fp8mlp_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         missing = [name for name in EXPORTS if not hasattr(L, name)]
@@ -195,6 +204,23 @@ def fp8mlp_gemm_fp8(M: int, N: int, K: int, A, a_kmajor: bool, a_fmt: int, B, b_
                     scale_a, scale_b, out) -> None:
     _check(lib().fp8mlp_gemm_fp8(M, N, K, _ptr(A), int(a_kmajor), a_fmt, _ptr(B), int(b_kmajor), b_fmt,
                                  _ptr(scale_a), _ptr(scale_b), _ptr(out), _stream()), "fp8mlp_gemm_fp8")
+
+
+def fp8mlp_adam_step(tensors: list, lr: float, beta1: float, beta2: float, eps: float, weight_decay: float,
+                     step: int) -> None:
+    """tensors: dicts with torch tensors w, g (fp32), m, v (uint8 codes) and 1-element fp32 tensors
+    scale_m_in, scale_v_in, scale_m_out, scale_v_out, amax_m, amax_v.  Everything is updated in place."""
+    arr = (_AdamTensor * len(tensors))()
+    for a, t in zip(arr, tensors):
+        a.w, a.g, a.m, a.v, a.n = t["w"].data_ptr(), t["g"].data_ptr(), t["m"].data_ptr(), t["v"].data_ptr(), t["w"].numel()
+        for k in ("scale_m_in", "scale_v_in", "scale_m_out", "scale_v_out", "amax_m", "amax_v"):
+            setattr(a, k, t[k].data_ptr())
+    _check(lib().fp8mlp_adam_step(arr, len(tensors), lr, beta1, beta2, eps, weight_decay, step, _stream()),
+           "fp8mlp_adam_step")
+
+
+def fp8mlp_scale_from_amax(amax, fp8_fmt: int, scale) -> None:
+    _check(lib().fp8mlp_scale_from_amax(_ptr(amax), fp8_fmt, _ptr(scale), _stream()), "fp8mlp_scale_from_amax")
 
 
 # ---------------------------------------------------------------- conveniences (allocation only)

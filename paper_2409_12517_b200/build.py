@@ -9,7 +9,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libfp8mlp.so"
-SOURCES = ["api.cu", "gemm.cu", "quantize.cu"]
+SOURCES = ["api.cu", "gemm.cu", "quantize.cu", "adam.cu"]
 HEADERS = ["common.cuh", "gemm.cuh", "quantize.cuh", "../../include/fp8mlp.h"]
 
 NVCC_FLAGS = [

@@ -308,6 +308,12 @@ int fp8mlp_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, 
                              amax, sms, st);
 }
 
+int fp8mlp_scale_from_amax(const float* amax, int fp8_fmt, float* scale, void* stream) {
+    if (amax == nullptr || scale == nullptr) return FP8MLP_ERR_ARG;
+    if (fp8_fmt != FP8MLP_E4M3 && fp8_fmt != FP8MLP_E5M2) return FP8MLP_ERR_ARG;
+    return run_scale_from_amax(fp8_fmt, amax, nullptr, scale, static_cast<cudaStream_t>(stream));
+}
+
 int fp8mlp_update_scales(fp8mlp_ctx* c, const fp8mlp_amax* am, fp8mlp_scales* sc, void* stream) {
     if (c == nullptr || am == nullptr || sc == nullptr) return FP8MLP_ERR_ARG;
     UpdateScalesArgs a{};

@@ -275,6 +275,11 @@ __device__ __forceinline__ void ld_global_nc_v8(const void* p, uint32_t (&w)[8])
                  : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
                  : "l"(p));
 }
+__device__ __forceinline__ void ld_global_v8(const void* p, uint32_t (&w)[8]) {     // data the kernel also writes
+    asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p) : "memory");
+}
 __device__ __forceinline__ uint4 ld_global_nc_v4(const void* p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0, %1, %2, %3}, [%4];"
