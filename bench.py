@@ -264,6 +264,29 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps, world, "cuda")
+    # the step after backward (not part of the metric): Adam with FP8 moments on W1, W2, W3 from dW1, dW2, dW3
+    adam = None
+    if rank == 0:
+        one = lambda: torch.ones(1, device="cuda")
+        states = [dict(w=W.view(-1), g=dW.view(-1), m=torch.zeros(W.numel(), dtype=torch.uint8, device="cuda"),
+                       v=torch.zeros(W.numel(), dtype=torch.uint8, device="cuda"), scale_m_in=one(), scale_v_in=one(),
+                       scale_m_out=one(), scale_v_out=one(), amax_m=torch.zeros(1, device="cuda"),
+                       amax_v=torch.zeros(1, device="cuda")) for W, dW in ((W1, dW1), (W2, dW2), (W3, dW3))]
+        hp = dict(lr=0.0, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.0)      # lr 0: the weights stay put
+        for t in range(1, 4):
+            B.fp8mlp_adam_step(states, step=t, **hp)
+        torch.cuda.synchronize()
+        n_adam = 20
+        e0.record()
+        for t in range(4, 4 + n_adam):
+            B.fp8mlp_adam_step(states, step=t, **hp)
+        e1.record()
+        torch.cuda.synchronize()
+        adam_ms = e0.elapsed_time(e1) / n_adam
+        adam_bytes = 16.0 * 3 * d * f                # g 4 + w 4+4 + codes 1+1+1+1 per parameter
+        adam = {"ms": round(adam_ms, 4), "params": 3 * d * f, "bytes_per_param": 16,
+                "gbs": round(adam_bytes / (adam_ms * 1e-3) / 1e9, 1)}
+        del states
     B.fp8mlp_destroy(ctx)
     if rank != 0:
         return
@@ -316,6 +339,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "roofline": roofline,
         "kernels": kernels,
     }
+    if adam is not None:
+        adam["frac_of_hbm_peak"] = round(adam["gbs"] / peaks["hbm_gbs"], 3)
+        out["after_the_step"] = {"adam_fp8_moments": adam,
+                                 "note": "Adam with E4M3/E5M2 moments on W1, W2, W3; not included in value"}
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(out))
