@@ -168,6 +168,23 @@ FP8MLP_API int fp8mlp_backward(fp8mlp_ctx* ctx, int64_t T, const void* dy_bf16,
                     int scale_mode, fp8mlp_scales* scales, fp8mlp_amax* amax,
                     void* dx_bf16, float* dW1, float* dW2, float* dW3, void* stream);
 
+/* Inference form of Smooth-SwiGLU (end of Section 4.4): once s_i is fixed it is folded into the weights,
+ *   w1~_i = Q(s_i w1_i),   w3~_i = Q(s_i^-1 w3_i),
+ * and the block becomes an ordinary FP8 SwiGLU MLP on the merged weights with one per-tensor scale for the
+ * SwiGLU output - the per-channel scaling costs nothing at run time.
+ * fp8mlp_merge_weights quantises [W2 | W1 diag(s)] (one scale, scales.w12) and diag(1/s) W3 (scales.w3) into the
+ * context, once; s[f] device floats.  SCALE_GIVEN reads the two scales, SCALE_FROM_CURRENT_AMAX derives them
+ * (amax.w1 = max |W1 diag(s)|, amax.w2, amax.w3 = max |diag(1/s) W3|; `amax` and its members nullable).
+ * fp8mlp_forward_merged then runs  Xq = Q(x sx);  G = Xq W2q, U~ = Xq W1~q (dequantised);  H~ = U~ G sigma(G);
+ * Hq = Q(H~ sh);  Y = Hq W3~q / (sw3 sh)  with sh = scales.h[0] (scales.h[f] holds sh repeated, as with
+ * Smooth off).  SCALE_FROM_CURRENT_AMAX derives sx and sh from this call's data (amax.x, amax.h[f] required);
+ * with SCALE_GIVEN amax and its members are optional and the per-channel maxima are only computed if amax.h is
+ * given.  FP8MLP_ERR_STATE unless the context holds merged weights (fp8mlp_forward replaces them). */
+FP8MLP_API int fp8mlp_merge_weights(fp8mlp_ctx* ctx, const float* W1, const float* W2, const float* W3, const float* s,
+                                    int scale_mode, fp8mlp_scales* scales, fp8mlp_amax* amax, void* stream);
+FP8MLP_API int fp8mlp_forward_merged(fp8mlp_ctx* ctx, int64_t T, const void* x_bf16, int scale_mode,
+                                     fp8mlp_scales* scales, fp8mlp_amax* amax, void* y_bf16, void* stream);
+
 /* Adam step with both moments stored in FP8 (Section 5: first moment E4M3, second moment E5M2 -
  * the update divides by the square root of the second moment, so its smallest values matter and it
  * needs the wider exponent range).  The step after fp8mlp_backward: it consumes dW1, dW2, dW3.

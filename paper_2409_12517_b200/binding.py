@@ -28,6 +28,7 @@ EXPORTS = [
     "fp8mlp_workspace", "fp8mlp_launch_count", "fp8mlp_quantize", "fp8mlp_update_scales",
     "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8", "fp8mlp_profile_enable", "fp8mlp_profile_read",
     "fp8mlp_forward_static", "fp8mlp_adam_step", "fp8mlp_scale_from_amax",
+    "fp8mlp_merge_weights", "fp8mlp_forward_merged",
 ]
 PHASES = ["quant_x", "quant_w12", "quant_w3", "gemm1_swiglu", "gemm2_down", "quant_dy", "dgrad2_swiglu_bwd",
           "wgrad3", "dgrad1", "wgrad12", "misc"]
@@ -86,6 +87,10 @@ def lib():
         L.fp8mlp_forward_static.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_uint32, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_int, C.POINTER(_Scales), C.POINTER(_Amax),
                                             C.c_void_p, C.c_void_p]
+        L.fp8mlp_merge_weights.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                           C.POINTER(_Scales), C.POINTER(_Amax), C.c_void_p]
+        L.fp8mlp_forward_merged.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int, C.POINTER(_Scales),
+                                            C.POINTER(_Amax), C.c_void_p, C.c_void_p]
         L.fp8mlp_adam_step.argtypes = [C.POINTER(_AdamTensor), C.c_int, C.c_float, C.c_float, C.c_float, C.c_float,
                                        C.c_float, C.c_int64, C.c_void_p]
         L.fp8mlp_scale_from_amax.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
@@ -204,6 +209,18 @@ def fp8mlp_gemm_fp8(M: int, N: int, K: int, A, a_kmajor: bool, a_fmt: int, B, b_
                     scale_a, scale_b, out) -> None:
     _check(lib().fp8mlp_gemm_fp8(M, N, K, _ptr(A), int(a_kmajor), a_fmt, _ptr(B), int(b_kmajor), b_fmt,
                                  _ptr(scale_a), _ptr(scale_b), _ptr(out), _stream()), "fp8mlp_gemm_fp8")
+
+
+def fp8mlp_merge_weights(ctx: int, W1, W2, W3, s, scale_mode: int, scales: dict, amax: dict | None) -> None:
+    sc, a = _scales(scales), _amax(amax)
+    _check(lib().fp8mlp_merge_weights(C.c_void_p(ctx), _ptr(W1), _ptr(W2), _ptr(W3), _ptr(s), scale_mode, C.byref(sc),
+                                      C.byref(a) if a is not None else None, _stream()), "fp8mlp_merge_weights")
+
+
+def fp8mlp_forward_merged(ctx: int, T: int, x, scale_mode: int, scales: dict, amax: dict | None, y) -> None:
+    sc, a = _scales(scales), _amax(amax)
+    _check(lib().fp8mlp_forward_merged(C.c_void_p(ctx), T, _ptr(x), scale_mode, C.byref(sc),
+                                       C.byref(a) if a is not None else None, _ptr(y), _stream()), "fp8mlp_forward_merged")
 
 
 def fp8mlp_adam_step(tensors: list, lr: float, beta1: float, beta2: float, eps: float, weight_decay: float,

@@ -46,6 +46,7 @@ struct fp8mlp_ctx {
     float* dummy;     // [8 + f] sinks for amax outputs the caller did not ask for
     int* status;      // bounded-wait status word
     int64_t saved_T;  // tokens of the last forward that saved activations, -1 if none
+    bool merged;      // the FP8 weights hold the inference-merged form (fp8mlp_merge_weights)
     int64_t bytes[7];
     // per-phase timing
     bool profiling;
@@ -150,7 +151,8 @@ int quantize_w12(fp8mlp_ctx* c, const float* W1, const float* W2, int mode, floa
 }
 
 // G|U = Xq [W2q|W1q] with the SwiGLU / Smooth-SwiGLU epilogue
-int gemm1_swiglu(fp8mlp_ctx* c, int64_t T, const fp8mlp_scales* s, float* amax_h, int store, cudaStream_t st) {
+int gemm1_swiglu(fp8mlp_ctx* c, int64_t T, const fp8mlp_scales* s, float* amax_h, int store, cudaStream_t st,
+                 bool save_gu = true) {
     CUtensorMap tmA, tmB0, tmB1;
     FP8MLP_TRY(make_tmap_u8(&tmA, c->xq, c->d, T, c->d));
     FP8MLP_TRY(make_tmap_u8(&tmB0, c->w12q, c->f, c->d, 2 * c->f));
@@ -162,7 +164,7 @@ int gemm1_swiglu(fp8mlp_ctx* c, int64_t T, const fp8mlp_scales* s, float* amax_h
     a.s_h = s->h;
     a.store = store;
     a.hq = c->hq;
-    a.gu = (c->flags & FP8MLP_SAVE_FOR_BWD) ? c->gu : nullptr;
+    a.gu = (save_gu && (c->flags & FP8MLP_SAVE_FOR_BWD)) ? c->gu : nullptr;
     a.amax_h = reinterpret_cast<unsigned int*>(amax_h);
     return launch_gemm(EPI_SWIGLU_FWD, false, true, FP8MLP_E4M3, FP8MLP_E4M3, tmA, tmB0, tmB1, a, c->sm_count, st);
 }
@@ -347,6 +349,7 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
     float* a_w3 = (am && am->w3) ? am->w3 : c->dummy + 3;
     float* a_h = (am && am->h) ? am->h : c->dummy + 8;
     c->saved_T = -1;
+    c->merged = false;
 
     {
         PhaseTimer pt(c, FP8MLP_PH_MISC, st);
@@ -404,6 +407,86 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
     FP8MLP_TRY(launch_gemm(EPI_BF16, false, true, FP8MLP_E4M3, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
     if (c->flags & FP8MLP_SAVE_FOR_BWD) c->saved_T = T;
     return FP8MLP_OK;
+}
+
+int fp8mlp_merge_weights(fp8mlp_ctx* c, const float* W1, const float* W2, const float* W3, const float* s,
+                         int mode, fp8mlp_scales* sc, fp8mlp_amax* am, void* stream) {
+    if (c == nullptr || sc == nullptr || W1 == nullptr || W2 == nullptr || W3 == nullptr || s == nullptr) return FP8MLP_ERR_ARG;
+    if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
+    if (sc->w12 == nullptr || sc->w3 == nullptr) return FP8MLP_ERR_ARG;
+    if (!aligned16(W1) || !aligned16(W2) || !aligned16(W3) || !aligned16(s)) return FP8MLP_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t d = c->d, f = c->f;
+    float* a_w1 = (am && am->w1) ? am->w1 : c->dummy + 1;
+    float* a_w2 = (am && am->w2) ? am->w2 : c->dummy + 2;
+    float* a_w3 = (am && am->w3) ? am->w3 : c->dummy + 3;
+    c->saved_T = -1;
+    c->merged = false;
+    FP8MLP_TRY(zero_floats({a_w1, a_w2, a_w3}, st));
+    QuantTensor t[3] = {};
+    t[0].src = W2; t[0].rows = d; t[0].cols = f; t[0].dst = c->w12q; t[0].ld_dst = 2 * f; t[0].amax = a_w2;
+    t[1].src = W1; t[1].rows = d; t[1].cols = f; t[1].dst = c->w12q + f; t[1].ld_dst = 2 * f; t[1].amax = a_w1;
+    t[1].col_mul = s;                                            // w1~_i = s_i w1_i
+    t[2].src = W3; t[2].rows = f; t[2].cols = d; t[2].dst = c->w3q; t[2].ld_dst = d; t[2].amax = a_w3;
+    t[2].row_div = s; t[2].scale = sc->w3;                       // w3~_i = s_i^-1 w3_i
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
+        FP8MLP_TRY(run_quantize_segments(false, true, FP8MLP_F32, FP8MLP_E4M3, t, 3, nullptr, c->sm_count, st));
+        FP8MLP_TRY(run_scale_from_amax(FP8MLP_E4M3, a_w1, a_w2, sc->w12, st));
+        FP8MLP_TRY(run_scale_from_amax(FP8MLP_E4M3, a_w3, nullptr, sc->w3, st));
+        FP8MLP_TRY(run_quantize_segments(true, false, FP8MLP_F32, FP8MLP_E4M3, t, 3, sc->w12, c->sm_count, st));
+    } else {
+        FP8MLP_TRY(run_quantize_segments(true, true, FP8MLP_F32, FP8MLP_E4M3, t, 3, sc->w12, c->sm_count, st));
+    }
+    c->merged = true;
+    return FP8MLP_OK;
+}
+
+int fp8mlp_forward_merged(fp8mlp_ctx* c, int64_t T, const void* x, int mode, fp8mlp_scales* sc, fp8mlp_amax* am,
+                          void* y, void* stream) {
+    if (c == nullptr || sc == nullptr) return FP8MLP_ERR_ARG;
+    if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
+    if (T < 0 || T > c->T_max) return FP8MLP_ERR_SHAPE;
+    if (!c->merged) return FP8MLP_ERR_STATE;
+    if (T > 0 && (x == nullptr || y == nullptr)) return FP8MLP_ERR_ARG;
+    if (sc->x == nullptr || sc->w12 == nullptr || sc->w3 == nullptr || sc->h == nullptr) return FP8MLP_ERR_ARG;
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX && (am == nullptr || am->x == nullptr || am->h == nullptr)) return FP8MLP_ERR_ARG;
+    if (!aligned16(x) || !aligned16(y)) return FP8MLP_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t d = c->d, f = c->f;
+    float* a_x = (am && am->x) ? am->x : c->dummy + 0;
+    float* a_h = (am && am->h) ? am->h : nullptr;                // maxima of H only if asked for
+    if (T == 0) return FP8MLP_OK;
+    {
+        PhaseTimer pt(c, FP8MLP_PH_MISC, st);
+        FP8MLP_TRY(zero_floats({a_x}, st, a_h, f));
+    }
+    {
+        PhaseTimer pt(c, FP8MLP_PH_QUANT_X, st);
+        FP8MLP_TRY(quantize_tensor(x, FP8MLP_BF16, T, d, FP8MLP_E4M3, mode, sc->x, a_x, nullptr, nullptr, nullptr, c->xq, d, c->sm_count, st));
+    }
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
+        {
+            PhaseTimer pt(c, FP8MLP_PH_GEMM1, st);
+            FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/0, st, /*save_gu=*/false));
+        }
+        PhaseTimer pt(c, FP8MLP_PH_MISC, st);
+        UpdateScalesArgs u{};
+        u.amax_h = a_h; u.scale_h = sc->h; u.f = f; u.smooth = 0;   // one per-tensor scale: the s_i sit in the weights
+        FP8MLP_TRY(run_update_scales(u, c->sm_count, st));
+    }
+    {
+        PhaseTimer pt(c, FP8MLP_PH_GEMM1, st);
+        FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/1, st, /*save_gu=*/false));
+    }
+    PhaseTimer pt2(c, FP8MLP_PH_GEMM2, st);
+    CUtensorMap tmA, tmB;
+    FP8MLP_TRY(make_tmap_u8(&tmA, c->hq, f, T, f));
+    FP8MLP_TRY(make_tmap_u8(&tmB, c->w3q, d, f, d));
+    GemmArgs a = base_args(c, static_cast<int>(T), static_cast<int>(d), static_cast<int>(f));
+    a.s0 = sc->w3;
+    a.s1 = sc->h;
+    a.out_bf16 = static_cast<uint16_t*>(y);
+    return launch_gemm(EPI_BF16, false, true, FP8MLP_E4M3, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st);
 }
 
 int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_scales* sc, fp8mlp_amax* am,

@@ -196,13 +196,15 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
         for (int e = 0; e < 32; ++e) h[e] = rcp_approx(__fadd_rn(1.0f, h[e]));          // sigma(G)
 #pragma unroll
         for (int e = 0; e < 32; ++e) h[e] = __fmul_rn(u[e], __fmul_rn(g[e], h[e]));       // H
-        float colmax = 0.0f;
+        if (p.amax_h != nullptr) {
+            float colmax = 0.0f;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            const float cm = warp_max_nonneg(fabsf(h[e]));       // max over this warp's 32 rows
-            if (lane == e) colmax = cm;
+            for (int e = 0; e < 32; ++e) {
+                const float cm = warp_max_nonneg(fabsf(h[e]));   // max over this warp's 32 rows
+                if (lane == e) colmax = cm;
+            }
+            atomicMax(&tail->amax_tile[32 * j + lane], __float_as_uint(colmax));
         }
-        atomicMax(&tail->amax_tile[32 * j + lane], __float_as_uint(colmax));
         if (!p.store || !row_ok) continue;
         const bool both = c0 + 16 < f;
         if (p.gu != nullptr) {
@@ -478,7 +480,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             if constexpr (EPI == EPI_SWIGLU_FWD) {
                 epi_bar_sync();                        // all eight warps have merged into amax_tile
-                if (et < 128) {
+                if (et < 128 && p.amax_h != nullptr) {
                     const unsigned int v = tail->amax_tile[et];
                     if ((n0 + et) < p.N && v != 0u) atomicMax(p.amax_h + n0 + et, v);
                 }

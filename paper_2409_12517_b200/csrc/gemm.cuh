@@ -59,7 +59,7 @@ struct GemmArgs {
     int wide;               // outputs may be written 32 bytes at a time (rows and bases 32-byte aligned)
     uint8_t* hq;            // fwd: E4M3 [M, f]
     uint16_t* gu;           // fwd: out (nullable), bwd: in; bf16 [M, 2f] = G | U
-    unsigned int* amax_h;   // fwd: [f] bit patterns of max |H|, raised atomically
+    unsigned int* amax_h;   // fwd: [f] bit patterns of max |H|, raised atomically; null: maxima not wanted
     const float* sdz;       // bwd: scale of dZ
     uint8_t* dzq;           // bwd: E5M2 [M, 2f] = dG | dU
     unsigned int* amax_dz;  // bwd: bit pattern of max(|dG|, |dU|), raised atomically

@@ -100,7 +100,7 @@ quantize_kernel(const QuantLaunch q) {
     const uint32_t begin = (blockIdx.x / q.nseg) * q.units_per_block;
     const uint32_t end = min(begin + q.units_per_block, sg.n_units);
     const bool has_row = sg.row_mul != nullptr || sg.row_div != nullptr;
-    const bool flat = !has_row && sg.ld_dst == static_cast<int64_t>(sg.units_per_row) * E;
+    const bool flat = !has_row && sg.col_mul == nullptr && sg.ld_dst == static_cast<int64_t>(sg.units_per_row) * E;
     // (row, column unit) of this thread's next unit, advanced by kThreads units at a time: one
     // division per thread instead of one per unit
     const uint32_t upr = sg.units_per_row;
@@ -138,6 +138,11 @@ quantize_kernel(const QuantLaunch q) {
 #pragma unroll
                     for (int i = 0; i < E; ++i) v[i] = __fmul_rn(v[i], m);
                 }
+            }
+            if (sg.col_mul != nullptr) {
+                const float* cm = sg.col_mul + static_cast<int64_t>(col[k]) * E;
+#pragma unroll
+                for (int i = 0; i < E; ++i) v[i] = __fmul_rn(v[i], cm[i]);
             }
             if constexpr (AMAX) {
 #pragma unroll
@@ -249,7 +254,7 @@ int run_quantize_segments(bool cast, bool amax, int src_dtype, int fmt, const Qu
     for (int i = 0; i < nseg; ++i) {
         QuantSeg& sg = q.seg[i];
         sg.src = t[i].src; sg.dst = t[i].dst; sg.amax = t[i].amax;
-        sg.row_mul = t[i].row_mul; sg.row_div = t[i].row_div;
+        sg.row_mul = t[i].row_mul; sg.row_div = t[i].row_div; sg.col_mul = t[i].col_mul;
         sg.scale = t[i].scale != nullptr ? t[i].scale : scale;
         sg.units_per_row = static_cast<uint32_t>(t[i].cols / elems);
         sg.n_units = static_cast<uint32_t>(t[i].rows * (t[i].cols / elems));

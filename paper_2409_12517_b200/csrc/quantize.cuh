@@ -16,11 +16,13 @@ struct QuantTensor {
     float* amax;            // raised atomically to max |src * multiplier| (amax passes; zeroed by the caller)
     const float* row_mul;   // nullable: row r is multiplied by row_mul[r] first
     const float* row_div;   // nullable: row r is multiplied by 1 / row_div[r] first (W3' = diag(s^-1) W3)
+    const float* col_mul;   // nullable: column c is multiplied by col_mul[c] first (merged w1~ = s_i w1_i)
     const float* scale;     // nullable: overrides the launch's scale for this tensor
 };
 // what the kernel sees
 struct QuantSeg {
-    const void* src; uint8_t* dst; float* amax; const float* row_mul; const float* row_div; const float* scale;
+    const void* src; uint8_t* dst; float* amax; const float* row_mul; const float* row_div; const float* col_mul;
+    const float* scale;
     int64_t ld_dst; uint32_t units_per_row, n_units;
 };
 struct QuantLaunch { QuantSeg seg[kMaxQuantSegs]; int nseg; int wide; uint32_t units_per_block; const float* scale; };
