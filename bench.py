@@ -306,6 +306,30 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         merged = {"ms": round(inf_ms, 4), "tflops": round(6.0 * T * d * f / (inf_ms * 1e-3) / 1e12, 1),
                   "what": "quantise x + gate/up GEMM with SwiGLU epilogue + down GEMM on merged FP8 weights"}
     B.fp8mlp_destroy(ctx)
+    # the same step with plain per-tensor FP8 for the SwiGLU output (Smooth-SwiGLU off), for the cost of smoothing
+    plain = None
+    if rank == 0:
+        ctx0 = B.fp8mlp_create(T, d, f, B.SAVE_FOR_BWD)
+        sc0, am0 = B.new_scales(f), B.new_amax(f)
+
+        def step0(mode=B.SCALE_GIVEN):
+            B.fp8mlp_forward(ctx0, T, x, W1, W2, W3, mode, sc0, am0, y)
+            B.fp8mlp_backward(ctx0, T, dy, mode, sc0, am0, dx, dW1, dW2, dW3)
+
+        step0(B.SCALE_FROM_CURRENT_AMAX)
+        for _ in range(3):
+            step0()
+        torch.cuda.synchronize()
+        n0_steps = max(1, min(args.steps, 50))
+        e0.record()
+        for _ in range(n0_steps):
+            step0()
+        e1.record()
+        torch.cuda.synchronize()
+        assert B.fp8mlp_status(ctx0) == B.OK
+        plain_ms = e0.elapsed_time(e1) / n0_steps
+        plain = {"ms_per_step": round(plain_ms, 4), "tflops": round(job_tflops(T, d, f, 1, plain_ms), 1)}
+        B.fp8mlp_destroy(ctx0)
     if rank != 0:
         return
 
@@ -361,6 +385,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         adam["frac_of_hbm_peak"] = round(adam["gbs"] / peaks["hbm_gbs"], 3)
         merged["frac_of_fp8_peak"] = round(merged["tflops"] / fp8_peak, 3)
         out["beside_the_step"] = {"adam_fp8_moments": adam, "inference_merged_forward": merged,
+                                  "step_with_smooth_swiglu_off": plain,
                                   "note": "Adam with E4M3/E5M2 moments on W1, W2, W3, and the inference form of "
                                           "Smooth-SwiGLU; neither is included in value"}
     if world == 1 and not args.no_cpu_baseline:
