@@ -246,24 +246,51 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     xh, dyh = x.cpu().pin_memory(), dy.cpu().pin_memory()
     yh, dxh = torch.empty_like(xh).pin_memory(), torch.empty_like(xh).pin_memory()
 
-    def e2e_step():
-        x.copy_(xh, non_blocking=True)
-        B.fp8mlp_forward(ctx, T, x, W1, W2, W3, B.SCALE_GIVEN, sc, am, y)
-        yh.copy_(y, non_blocking=True)
-        dy.copy_(dyh, non_blocking=True)
-        B.fp8mlp_backward(ctx, T, dy, B.SCALE_GIVEN, sc, am, dx, dW1, dW2, dW3)
-        dxh.copy_(dx, non_blocking=True)
+    # Three streams, double-buffered device tensors: the copies of step i+1 (in) and step i-1 (out) run
+    # beside the kernels of step i.  Every step's inputs still come from host memory and its results
+    # still end in host memory inside the timed region.
+    main = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    xb, dyb = [x, torch.empty_like(x)], [dy, torch.empty_like(dy)]
+    yb, dxb = [y, torch.empty_like(y)], [dx, torch.empty_like(dx)]
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_comp = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
 
-    e2e_steps = max(1, min(args.steps, 10))
-    for _ in range(3):
-        e2e_step()
+    def e2e_run(n):
+        s_in.wait_stream(main)
+        s_out.wait_stream(main)
+        for i in range(n):
+            b = i & 1
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_comp[b])              # step i-2 has consumed this input buffer
+                xb[b].copy_(xh, non_blocking=True)
+                dyb[b].copy_(dyh, non_blocking=True)
+                ev_in[b].record(s_in)
+            main.wait_event(ev_in[b])
+            if i >= 2:
+                main.wait_event(ev_out[b])                   # step i-2's results have left this output buffer
+            B.fp8mlp_forward(ctx, T, xb[b], W1, W2, W3, B.SCALE_GIVEN, sc, am, yb[b])
+            B.fp8mlp_backward(ctx, T, dyb[b], B.SCALE_GIVEN, sc, am, dxb[b], dW1, dW2, dW3)
+            ev_comp[b].record(main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_comp[b])
+                yh.copy_(yb[b], non_blocking=True)
+                dxh.copy_(dxb[b], non_blocking=True)
+                ev_out[b].record(s_out)
+        main.wait_stream(s_out)
+        main.wait_stream(s_in)
+
+    e2e_steps = max(4, min(args.steps, 20))
+    e2e_run(4)
     barrier()
     e0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
+    e2e_run(e2e_steps)
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps, world, "cuda")
+    del xb, dyb, yb, dxb
     # the step after backward (not part of the metric): Adam with FP8 moments on W1, W2, W3 from dW1, dW2, dW3
     adam = None
     if rank == 0:
@@ -376,7 +403,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "clocks": clocks,
         "e2e": {"value": round(job_tflops(T, d, f, world, e2e_ms), 2), "unit": UNIT,
                 "ms_per_step": round(e2e_ms, 4), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "what": "x and dY copied from pinned host memory, Y and dX copied back, weights resident"},
+                "what": "every step: x and dY copied from pinned host memory, Y and dX copied back to it; copies "
+                        "on their own streams overlap the neighbouring steps' kernels; weights resident"},
         "gpu_launches": launches,
         "roofline": roofline,
         "kernels": kernels,
