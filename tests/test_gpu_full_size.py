@@ -95,7 +95,8 @@ def _sample(rng, n, count, always=()):
 
 
 @pytest.mark.parametrize("name,smooth,n_prev,n_tok,n_ch", [("7b", True, 48, 24, 32), ("7b", False, 32, 12, 24),
-                                                            ("70b", True, 16, 8, 20)])
+                                                            ("70b", True, 16, 8, 20),
+                                                            ("sweep_32768", True, 32, 12, 12)])   # largest T, x50 token rows
 def test_full_size_sampled_parity(name, smooth, n_prev, n_tok, n_ch):
     w = wl.make_config(name)
     T, d, f = w.T, w.d, w.f
