@@ -20,7 +20,7 @@ _ADAM_SRC = _HERE / "fp8adam_oracle.c"
 _ADAM_LIB = _HERE / "liboracle_adam.so"
 
 E4M3, E5M2 = 0, 1
-FLAG_SMOOTH, FLAG_Q_IDENTITY, FLAG_NO_BF16 = 1, 2, 4
+FLAG_SMOOTH, FLAG_Q_IDENTITY, FLAG_NO_BF16, FLAG_H_BF16 = 1, 2, 4, 8
 SCALE_GIVEN, SCALE_CURRENT = 0, 1
 
 _lib = None

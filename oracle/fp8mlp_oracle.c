@@ -48,6 +48,9 @@
 #define ORC_FLAG_SMOOTH      1u  /* per-channel s_i (Eq. 2); otherwise one per-tensor scale for H */
 #define ORC_FLAG_Q_IDENTITY  2u  /* Q(v) = v: skip the FP8 rounding (pins only)                  */
 #define ORC_FLAG_NO_BF16     4u  /* keep G, U, Y, dX in fp32 instead of rounding to bf16 (pins)  */
+#define ORC_FLAG_H_BF16      8u  /* the paper's "SwiGLU output in BF16" variant (Section 4.3): the
+                                    last linear layer is not quantised - its input H, its weight W3
+                                    and the dY it meets in backward are bf16; everything else FP8   */
 
 #define ORC_SCALE_GIVEN   0
 #define ORC_SCALE_CURRENT 1
@@ -359,6 +362,16 @@ int orc_forward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode,
         }
     }
     /* Q(s_i * H) (Eq. 2) */
+    const int h_bf16 = (flags & ORC_FLAG_H_BF16) != 0;
+    if (h_bf16) {
+        /* READING: "disabling the quantisation of the last linear layer" = that layer runs in bf16:
+         * H and W3 are rounded to bf16 (no scales), products accumulate in fp32. */
+        for (int64_t i = 0; i < f; ++i) s_h[i] = 1.0f;
+        for (int64_t i = 0; i < T * f; ++i) {
+            hq[i] = orc_bf16_to_f32(orc_f32_to_bf16(H[i]));
+            if (Hq) Hq[i] = 0;
+        }
+    } else
     for (int64_t t = 0; t < T; ++t)
         for (int64_t i = 0; i < f; ++i) {
             uint8_t code;
@@ -368,7 +381,14 @@ int orc_forward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode,
 
     /* W3' = diag(s^-1) W3 and its quantisation (the merge of Section 4.4) */
     float dq2;
-    if (smooth) {
+    if (h_bf16) {
+        float a3 = orc_amax(W3, f * d);
+        for (int64_t i = 0; i < f * d; ++i) w3q[i] = orc_bf16_to_f32(orc_f32_to_bf16(W3[i]));
+        if (W3q) memset(W3q, 0, (size_t)(f * d));
+        if (amax_w3) *amax_w3 = a3;
+        *sw3 = 1.0f;
+        dq2 = 1.0f;
+    } else if (smooth) {
         for (int64_t i = 0; i < f; ++i) rmul[i] = 1.0f / s_h[i];
         float a3 = orc_amax_rows(W3, f, d, rmul);
         if (scale_mode == ORC_SCALE_CURRENT) *sw3 = orc_scale_from_amax(ORC_E4M3, a3);
@@ -444,6 +464,7 @@ int orc_backward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode
     float* acc  = (float*)malloc(sizeof(float) * (f * d > d * 2 * f ? f * d : d * 2 * f));
     if (!dyf || !dyq || !xq || !w12q || !w3q || !hq || !accH || !dG || !dU || !dzq || !accX || !acc) return -1;
 
+    const int h_bf16 = (flags & ORC_FLAG_H_BF16) != 0;
     if (qid) {
         memcpy(xq, xq_f, sizeof(float) * T * d);
         memcpy(w12q, w12q_f, sizeof(float) * d * 2 * f);
@@ -452,15 +473,26 @@ int orc_backward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode
     } else {
         orc_decode_array(ORC_E4M3, Xq, T * d, xq);
         orc_decode_array(ORC_E4M3, W12q, d * 2 * f, w12q);
-        orc_decode_array(ORC_E4M3, W3q, f * d, w3q);
-        orc_decode_array(ORC_E4M3, Hq, T * f, hq);
+        if (h_bf16) {                       /* the bf16 operands of the unquantised last layer */
+            memcpy(w3q, w3q_f, sizeof(float) * f * d);
+            memcpy(hq, hq_f, sizeof(float) * T * f);
+        } else {
+            orc_decode_array(ORC_E4M3, W3q, f * d, w3q);
+            orc_decode_array(ORC_E4M3, Hq, T * f, hq);
+        }
     }
 
     /* quantise dY (E5M2) */
     orc_bf16_to_f32_array(dy_bf16, T * d, dyf);
     float ady = orc_amax(dyf, T * d);
+    if (h_bf16) {                           /* dY only meets the bf16 layer: used as it is */
+        *sdy = 1.0f;
+        memcpy(dyq, dyf, sizeof(float) * T * d);
+        if (dYq) memset(dYq, 0, (size_t)(T * d));
+    } else {
     if (scale_mode == ORC_SCALE_CURRENT) *sdy = orc_scale_from_amax(ORC_E5M2, ady);
     orc_quantize(dyf, T, d, NULL, ORC_E5M2, *sdy, flags, dYq, d, dyq, NULL);
+    }
     if (amax_dy) *amax_dy = ady;
     const float inv_sdy = 1.0f / *sdy, inv_sw3 = 1.0f / sw3;
 

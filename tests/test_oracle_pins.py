@@ -389,3 +389,36 @@ def test_tiny_config_shapes_and_determinism():
     assert np.array_equal(o.W1[:, o.outlier_channels], np.float32(8) * o.W2[:, o.outlier_channels])
     t = wl.make("t", 4, 300, 16, 32, token_outlier_frac=0.01)
     assert t.outlier_tokens.size == 3
+
+
+# ---------------------------------------------------------------- "SwiGLU output in BF16" variant (Section 4.3)
+def test_h_bf16_variant_last_layer_runs_in_bf16():
+    """The paper's intermediate experiment: everything FP8 except the last linear layer of the block,
+    whose input (the SwiGLU output) is not quantised.  Pins: the layer's operands are the bf16
+    roundings a library produces; its outputs are the brute-force fp64 contractions of exactly those
+    operands; the variant sits closer to the unquantised block than plain FP8 when outlier channels
+    are present; and its gradients point where the fp64 block's do."""
+    import torch
+    w = wl.make("hb", 9, 48, 96, 208, w_std=0.05, channel_outlier_frac=0.02)
+    fl = oracle.FLAG_H_BF16
+    fw = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=fl | oracle.FLAG_NO_BF16, want_float_operands=True)
+    to_bf16 = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).to(torch.float32).numpy()
+    assert np.array_equal(fw["hq_f"], to_bf16(fw["H"])) and np.array_equal(fw["w3q_f"], to_bf16(w.W3))
+    assert fw["sw3"] == 1.0 and np.all(fw["s_h"] == 1.0)
+    Y_brute = fw["hq_f"].astype(np.float64) @ fw["w3q_f"].astype(np.float64)
+    assert np.abs(fw["Y"] - Y_brute).max() <= 1e-5 * np.abs(Y_brute).max()
+    bw = oracle.backward(fw, w.dY)
+    dy = wl.bf16_bits_to_f32(w.dY).astype(np.float64)
+    assert bw["sdy"] == 1.0
+    dW3_brute = fw["hq_f"].astype(np.float64).T @ dy
+    assert np.abs(bw["dW3"] - dW3_brute).max() <= 1e-5 * np.abs(dW3_brute).max()
+    # against the unquantised block
+    x = wl.bf16_bits_to_f32(w.x).astype(np.float64)
+    _, Y64 = oracle.mlp_f64(x, w.W1, w.W2, w.W3)
+    dX64, dW1_64, dW2_64, dW3_64 = oracle.mlp_f64_backward(x, w.W1, w.W2, w.W3, dy)
+    plain = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=oracle.FLAG_NO_BF16)
+    err = lambda a, b: np.abs(a - b).max() / np.abs(b).max()
+    assert err(fw["Y"], Y64) < err(plain["Y"], Y64)
+    cos = lambda a, b: float((a * b).sum() / np.sqrt((a * a).sum() * (b * b).sum()))
+    for got, ref in ((bw["dX"], dX64), (bw["dW1"], dW1_64), (bw["dW2"], dW2_64), (bw["dW3"], dW3_64)):
+        assert cos(got.astype(np.float64), ref) > 0.99
