@@ -334,9 +334,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                   "what": "quantise x + gate/up GEMM with SwiGLU epilogue + down GEMM on merged FP8 weights"}
     B.fp8mlp_destroy(ctx)
     # the same step with plain per-tensor FP8 for the SwiGLU output (Smooth-SwiGLU off), for the cost of smoothing
-    plain = None
-    if rank == 0:
-        ctx0 = B.fp8mlp_create(T, d, f, B.SAVE_FOR_BWD)
+    plain, hbf16 = None, None
+    for variant_flags in ((B.SAVE_FOR_BWD, B.H_BF16 | B.SAVE_FOR_BWD) if rank == 0 else ()):
+        ctx0 = B.fp8mlp_create(T, d, f, variant_flags)
         sc0, am0 = B.new_scales(f), B.new_amax(f)
 
         def step0(mode=B.SCALE_GIVEN):
@@ -354,8 +354,12 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         e1.record()
         torch.cuda.synchronize()
         assert B.fp8mlp_status(ctx0) == B.OK
-        plain_ms = e0.elapsed_time(e1) / n0_steps
-        plain = {"ms_per_step": round(plain_ms, 4), "tflops": round(job_tflops(T, d, f, 1, plain_ms), 1)}
+        v_ms = e0.elapsed_time(e1) / n0_steps
+        res = {"ms_per_step": round(v_ms, 4), "tflops": round(job_tflops(T, d, f, 1, v_ms), 1)}
+        if variant_flags & B.H_BF16:
+            hbf16 = res
+        else:
+            plain = res
         B.fp8mlp_destroy(ctx0)
     if rank != 0:
         return
@@ -414,8 +418,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         merged["frac_of_fp8_peak"] = round(merged["tflops"] / fp8_peak, 3)
         out["beside_the_step"] = {"adam_fp8_moments": adam, "inference_merged_forward": merged,
                                   "step_with_smooth_swiglu_off": plain,
+                                  "step_with_swiglu_output_in_bf16": hbf16,
                                   "note": "Adam with E4M3/E5M2 moments on W1, W2, W3, and the inference form of "
-                                          "Smooth-SwiGLU; neither is included in value"}
+                                          "Smooth-SwiGLU; the same step with plain per-tensor FP8 and with the last layer in "
+                                          "bf16 (the other rows of the paper's throughput table); none is included in value"}
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(out))

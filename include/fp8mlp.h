@@ -53,7 +53,10 @@ enum { FP8MLP_E4M3 = 0, FP8MLP_E5M2 = 1 };
 enum { FP8MLP_BF16 = 0, FP8MLP_F32 = 1 };
 enum {
     FP8MLP_SMOOTH = 1,       /* per-channel Smooth-SwiGLU scales; without it one per-tensor scale for H */
-    FP8MLP_SAVE_FOR_BWD = 2  /* forward keeps bf16 G = x W2 and U = x W1 for backward               */
+    FP8MLP_SAVE_FOR_BWD = 2, /* forward keeps bf16 G = x W2 and U = x W1 for backward               */
+    FP8MLP_H_BF16 = 4        /* the paper's "SwiGLU output in BF16" variant (Section 4.3): the last linear
+                                layer is not quantised - H, W3 and, in backward, dY are bf16 operands and
+                                scales.h / scales.w3 / scales.dy are unused; not with FP8MLP_SMOOTH        */
 };
 enum {
     FP8MLP_SCALE_GIVEN = 0,              /* delayed scaling: use the scale buffers as they are  */
@@ -66,7 +69,9 @@ enum { /* fp8mlp_workspace: internal buffers, for inspection by tests */
     FP8MLP_WS_HQ = 3,   /* E4M3 [T,f]   Q(s_i * SwiGLU)                                */
     FP8MLP_WS_GU = 4,   /* bf16 [T,2f]  saved G | U                                    */
     FP8MLP_WS_DYQ = 5,  /* E5M2 [T,d]   quantised dY                                   */
-    FP8MLP_WS_DZQ = 6   /* E5M2 [T,2f]  quantised [dG | dU]                            */
+    FP8MLP_WS_DZQ = 6,  /* E5M2 [T,2f]  quantised [dG | dU]                            */
+    FP8MLP_WS_HB = 7,   /* bf16 [T,f]   SwiGLU output, FP8MLP_H_BF16 contexts only      */
+    FP8MLP_WS_W3B = 8   /* bf16 [f,d]   W3 rounded to bf16, FP8MLP_H_BF16 contexts only */
 };
 
 enum { /* phases of one step, for fp8mlp_profile_read (SMOOTH-mode kernel sequence) */
@@ -263,6 +268,10 @@ FP8MLP_API int fp8mlp_gemm_fp8(int64_t M, int64_t N, int64_t K,
                     const uint8_t* A, int a_kmajor, int a_fmt,
                     const uint8_t* B, int b_kmajor, int b_fmt,
                     const float* scale_a, const float* scale_b, float* out, void* stream);
+
+/* The same for bf16 operands (the unquantised last layer of FP8MLP_H_BF16 contexts): A, B bf16, no scales. */
+FP8MLP_API int fp8mlp_gemm_bf16(int64_t M, int64_t N, int64_t K, const void* A, int a_kmajor, const void* B,
+                                int b_kmajor, float* out, void* stream);
 
 #ifdef __cplusplus
 }

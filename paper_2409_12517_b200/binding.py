@@ -19,16 +19,16 @@ OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_CUDA, ERR_TIMEOUT, ERR_STATE, ERR_TOO_LAR
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 E4M3, E5M2 = 0, 1
 BF16, F32 = 0, 1
-SMOOTH, SAVE_FOR_BWD = 1, 2
+SMOOTH, SAVE_FOR_BWD, H_BF16 = 1, 2, 4
 SCALE_GIVEN, SCALE_FROM_CURRENT_AMAX = 0, 1
-WS_XQ, WS_W12Q, WS_W3Q, WS_HQ, WS_GU, WS_DYQ, WS_DZQ = range(7)
+WS_XQ, WS_W12Q, WS_W3Q, WS_HQ, WS_GU, WS_DYQ, WS_DZQ, WS_HB, WS_W3B = range(9)
 
 EXPORTS = [
     "fp8mlp_create", "fp8mlp_destroy", "fp8mlp_strerror", "fp8mlp_last_cuda_error", "fp8mlp_status",
     "fp8mlp_workspace", "fp8mlp_launch_count", "fp8mlp_quantize", "fp8mlp_update_scales",
     "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8", "fp8mlp_profile_enable", "fp8mlp_profile_read",
     "fp8mlp_forward_static", "fp8mlp_adam_step", "fp8mlp_scale_from_amax",
-    "fp8mlp_merge_weights", "fp8mlp_forward_merged",
+    "fp8mlp_merge_weights", "fp8mlp_forward_merged", "fp8mlp_gemm_bf16",
 ]
 PHASES = ["quant_x", "quant_w12", "quant_w3", "gemm1_swiglu", "gemm2_down", "quant_dy", "dgrad2_swiglu_bwd",
           "wgrad3", "dgrad1", "wgrad12", "misc"]
@@ -87,6 +87,8 @@ def lib():
         L.fp8mlp_forward_static.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_uint32, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_int, C.POINTER(_Scales), C.POINTER(_Amax),
                                             C.c_void_p, C.c_void_p]
+        L.fp8mlp_gemm_bf16.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int, C.c_void_p, C.c_int,
+                                       C.c_void_p, C.c_void_p]
         L.fp8mlp_merge_weights.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                            C.POINTER(_Scales), C.POINTER(_Amax), C.c_void_p]
         L.fp8mlp_forward_merged.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int, C.POINTER(_Scales),
@@ -238,6 +240,11 @@ def fp8mlp_adam_step(tensors: list, lr: float, beta1: float, beta2: float, eps: 
 
 def fp8mlp_scale_from_amax(amax, fp8_fmt: int, scale) -> None:
     _check(lib().fp8mlp_scale_from_amax(_ptr(amax), fp8_fmt, _ptr(scale), _stream()), "fp8mlp_scale_from_amax")
+
+
+def fp8mlp_gemm_bf16(M: int, N: int, K: int, A, a_kmajor: bool, B, b_kmajor: bool, out) -> None:
+    _check(lib().fp8mlp_gemm_bf16(M, N, K, _ptr(A), int(a_kmajor), _ptr(B), int(b_kmajor), _ptr(out), _stream()),
+           "fp8mlp_gemm_bf16")
 
 
 # ---------------------------------------------------------------- conveniences (allocation only)

@@ -106,8 +106,14 @@ __global__ void __launch_bounds__(kAdamThreads, kAdamBlocksPerSm) adam_kernel(co
                 const float v = __fadd_rn(__fmul_rn(q.beta2, v_prev), __fmul_rn(q.omb2, __fmul_rn(g, g)));
                 const float mhat = __fmul_rn(m, q.c1);
                 const float vhat = __fmul_rn(v, q.c2);
-                const float den = __fadd_rn(__fsqrt_rn(vhat), q.eps);
-                float upd = __fdiv_rn(mhat, den);
+                // square root and division on the special-function unit (each within a few 2^-23 relative):
+                // correctly rounded versions cost ~25 more instructions per parameter, which at the clock
+                // the power cap leaves makes the pass instruction-bound instead of HBM-bound.  The moments
+                // and their codes do not depend on them; the weight moves by <= 1e-6 of its update.
+                float root, upd;
+                asm("sqrt.approx.f32 %0, %1;" : "=f"(root) : "f"(vhat));
+                const float den = __fadd_rn(root, q.eps);
+                asm("div.approx.f32 %0, %1, %2;" : "=f"(upd) : "f"(mhat), "f"(den));
                 if (q.wd != 0.0f) upd = __fadd_rn(upd, __fmul_rn(q.wd, w));
                 wn[i] = __float_as_uint(__fsub_rn(w, __fmul_rn(q.lr, upd)));
                 ms[i] = __fmul_rn(m, sm_out);

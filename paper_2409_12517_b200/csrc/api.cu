@@ -43,11 +43,12 @@ struct fp8mlp_ctx {
     int device, sm_count;
     uint8_t *xq, *w12q, *w3q, *hq, *dyq, *dzq;
     uint16_t* gu;
+    uint16_t *hb, *w3b;  // FP8MLP_H_BF16: the SwiGLU output and W3 in bf16 (operands of the unquantised last layer)
     float* dummy;     // [8 + f] sinks for amax outputs the caller did not ask for
     int* status;      // bounded-wait status word
     int64_t saved_T;  // tokens of the last forward that saved activations, -1 if none
     bool merged;      // the FP8 weights hold the inference-merged form (fp8mlp_merge_weights)
-    int64_t bytes[7];
+    int64_t bytes[9];
     // per-phase timing
     bool profiling;
     struct Bracket { int phase; cudaEvent_t e0, e1; };
@@ -164,6 +165,7 @@ int gemm1_swiglu(fp8mlp_ctx* c, int64_t T, const fp8mlp_scales* s, float* amax_h
     a.s_h = s->h;
     a.store = store;
     a.hq = c->hq;
+    a.hb = (c->flags & FP8MLP_H_BF16) ? c->hb : nullptr;
     a.gu = (save_gu && (c->flags & FP8MLP_SAVE_FOR_BWD)) ? c->gu : nullptr;
     a.amax_h = reinterpret_cast<unsigned int*>(amax_h);
     return launch_gemm(EPI_SWIGLU_FWD, false, true, FP8MLP_E4M3, FP8MLP_E4M3, tmA, tmB0, tmB1, a, c->sm_count, st);
@@ -194,7 +196,8 @@ int64_t fp8mlp_launch_count(void) { return g_launches.load(std::memory_order_rel
 int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_t flags) {
     if (out == nullptr) return FP8MLP_ERR_ARG;
     *out = nullptr;
-    if (flags & ~uint32_t(FP8MLP_SMOOTH | FP8MLP_SAVE_FOR_BWD)) return FP8MLP_ERR_ARG;
+    if (flags & ~uint32_t(FP8MLP_SMOOTH | FP8MLP_SAVE_FOR_BWD | FP8MLP_H_BF16)) return FP8MLP_ERR_ARG;
+    if ((flags & FP8MLP_SMOOTH) && (flags & FP8MLP_H_BF16)) return FP8MLP_ERR_ARG;   // nothing to smooth: H is not quantised
     if (T_max < 0 || d <= 0 || f <= 0 || d % 16 != 0 || f % 16 != 0) return FP8MLP_ERR_SHAPE;
     if (T_max > (1 << 30) || d > (1 << 24) || f > (1 << 24)) return FP8MLP_ERR_SHAPE;
     fp8mlp_ctx* c = new (std::nothrow) fp8mlp_ctx();
@@ -214,9 +217,17 @@ int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_
     c->bytes[FP8MLP_WS_GU] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * 2 * f * 2 : 16;
     c->bytes[FP8MLP_WS_DYQ] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * d : 16;
     c->bytes[FP8MLP_WS_DZQ] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * 2 * f : 16;
-    void** slots[7] = {(void**)&c->xq, (void**)&c->w12q, (void**)&c->w3q, (void**)&c->hq,
-                       (void**)&c->gu, (void**)&c->dyq, (void**)&c->dzq};
-    for (int i = 0; i < 7 && e == cudaSuccess; ++i) e = cudaMalloc(slots[i], static_cast<size_t>(c->bytes[i]));
+    const bool hb16 = (flags & FP8MLP_H_BF16) != 0;
+    if (hb16) {   // the last layer's operands are bf16: no FP8 copies of H, W3, dY
+        c->bytes[FP8MLP_WS_HQ] = 16;
+        c->bytes[FP8MLP_WS_W3Q] = 16;
+        c->bytes[FP8MLP_WS_DYQ] = 16;
+    }
+    c->bytes[FP8MLP_WS_HB] = hb16 ? Tm * f * 2 : 16;
+    c->bytes[FP8MLP_WS_W3B] = hb16 ? f * d * 2 : 16;
+    void** slots[9] = {(void**)&c->xq, (void**)&c->w12q, (void**)&c->w3q, (void**)&c->hq,
+                       (void**)&c->gu, (void**)&c->dyq, (void**)&c->dzq, (void**)&c->hb, (void**)&c->w3b};
+    for (int i = 0; i < 9 && e == cudaSuccess; ++i) e = cudaMalloc(slots[i], static_cast<size_t>(c->bytes[i]));
     if (e == cudaSuccess) e = cudaMalloc((void**)&c->dummy, sizeof(float) * (8 + f));
     if (e == cudaSuccess) e = cudaMalloc((void**)&c->status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int));
@@ -231,7 +242,7 @@ int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_
 
 int fp8mlp_destroy(fp8mlp_ctx* c) {
     if (c == nullptr) return FP8MLP_OK;
-    void* ptrs[] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq, c->dummy, c->status};
+    void* ptrs[] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq, c->hb, c->w3b, c->dummy, c->status};
     for (void* p : ptrs)
         if (p != nullptr) cudaFree(p);
     if (c->brackets != nullptr) {
@@ -282,8 +293,8 @@ int fp8mlp_profile_read(fp8mlp_ctx* c, double* ms, int64_t* count) {
 }
 
 int fp8mlp_workspace(fp8mlp_ctx* c, int which, void** ptr, int64_t* bytes) {
-    if (c == nullptr || ptr == nullptr || bytes == nullptr || which < 0 || which > FP8MLP_WS_DZQ) return FP8MLP_ERR_ARG;
-    void* all[7] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq};
+    if (c == nullptr || ptr == nullptr || bytes == nullptr || which < 0 || which > FP8MLP_WS_W3B) return FP8MLP_ERR_ARG;
+    void* all[9] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq, c->hb, c->w3b};
     *ptr = all[which];
     *bytes = c->bytes[which];
     return FP8MLP_OK;
@@ -359,6 +370,33 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
         PhaseTimer pt(c, FP8MLP_PH_QUANT_X, st);
         FP8MLP_TRY(quantize_tensor(x, FP8MLP_BF16, T, d, FP8MLP_E4M3, mode, sc->x, a_x, nullptr, nullptr, nullptr, c->xq, d, c->sm_count, st));
     }
+    if (c->flags & FP8MLP_H_BF16) {
+        // "SwiGLU output in BF16" variant: the last layer is not quantised.  [W2 | W1] -> E4M3, W3 -> bf16,
+        // GEMM-1 stores H in bf16 (no scale, so no calibration pass), GEMM-2 runs on bf16 operands.
+        {
+            PhaseTimer pt(c, FP8MLP_PH_QUANT_W12, st);
+            FP8MLP_TRY(quantize_w12(c, W1, W2, mode, sc->w12, a_w1, a_w2, st));
+        }
+        {
+            PhaseTimer pt(c, FP8MLP_PH_QUANT_W3, st);
+            FP8MLP_TRY(run_cast_bf16(W3, c->w3b, f * d, a_w3, c->sm_count, st));
+        }
+        if (T == 0) { c->saved_T = (c->flags & FP8MLP_SAVE_FOR_BWD) ? 0 : -1; return FP8MLP_OK; }
+        {
+            PhaseTimer pt(c, FP8MLP_PH_GEMM1, st);
+            FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/1, st));
+        }
+        PhaseTimer pt2(c, FP8MLP_PH_GEMM2, st);
+        CUtensorMap tmA, tmB;
+        FP8MLP_TRY(make_tmap(&tmA, c->hb, 2, false, f, T, 2 * f));
+        FP8MLP_TRY(make_tmap(&tmB, c->w3b, 2, true, d, f, 2 * d));
+        GemmArgs a = base_args(c, static_cast<int>(T), static_cast<int>(d), static_cast<int>(f));
+        a.elem_bytes = 2;
+        a.out_bf16 = static_cast<uint16_t*>(y);
+        FP8MLP_TRY(launch_gemm(EPI_BF16, false, true, 1, 1, tmA, tmB, tmB, a, c->sm_count, st));
+        if (c->flags & FP8MLP_SAVE_FOR_BWD) c->saved_T = T;
+        return FP8MLP_OK;
+    }
     if (mode == FP8MLP_SCALE_GIVEN) {
         // every scale is known: [W2 | W1] (one scale) and W3' = diag(1/s) W3 in one pass over the masters;
         // the reciprocal of s_i is taken inside the pass, row by row
@@ -414,6 +452,7 @@ int fp8mlp_merge_weights(fp8mlp_ctx* c, const float* W1, const float* W2, const 
     if (c == nullptr || sc == nullptr || W1 == nullptr || W2 == nullptr || W3 == nullptr || s == nullptr) return FP8MLP_ERR_ARG;
     if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
     if (sc->w12 == nullptr || sc->w3 == nullptr) return FP8MLP_ERR_ARG;
+    if (c->flags & FP8MLP_H_BF16) return FP8MLP_ERR_STATE;          // this context has no FP8 W3
     if (!aligned16(W1) || !aligned16(W2) || !aligned16(W3) || !aligned16(s)) return FP8MLP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t d = c->d, f = c->f;
@@ -517,7 +556,8 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
     }
     const int Ti = static_cast<int>(T), di = static_cast<int>(d), fi = static_cast<int>(f);
 
-    {   // dY -> E5M2
+    const bool hb16 = (c->flags & FP8MLP_H_BF16) != 0;
+    if (!hb16) {   // dY -> E5M2 (with the bf16 last layer dY is used as it is)
         PhaseTimer pt(c, FP8MLP_PH_QUANT_DY, st);
         FP8MLP_TRY(quantize_tensor(dy, FP8MLP_BF16, T, d, FP8MLP_E5M2, mode, sc->dy, a_dy, nullptr, nullptr, nullptr, c->dyq, d, c->sm_count, st));
     }
@@ -525,10 +565,18 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
     // dH~ = dYq W3q^T with the SwiGLU-backward epilogue -> dZq = [dG | dU]
     {
         CUtensorMap tmA, tmB;
-        FP8MLP_TRY(make_tmap_u8(&tmA, c->dyq, d, T, d));
-        FP8MLP_TRY(make_tmap_u8(&tmB, c->w3q, d, f, d));
         GemmArgs a = base_args(c, Ti, fi, di);
-        a.s0 = sc->dy; a.s1 = sc->w3;
+        int fa = FP8MLP_E5M2, fb = FP8MLP_E4M3;
+        if (hb16) {                      // dH = dY W3b^T on the bf16 operands, no dequantisation
+            FP8MLP_TRY(make_tmap(&tmA, dy, 2, false, d, T, 2 * d));
+            FP8MLP_TRY(make_tmap(&tmB, c->w3b, 2, false, d, f, 2 * d));
+            a.elem_bytes = 2;
+            fa = fb = 1;
+        } else {
+            FP8MLP_TRY(make_tmap_u8(&tmA, c->dyq, d, T, d));
+            FP8MLP_TRY(make_tmap_u8(&tmB, c->w3q, d, f, d));
+            a.s0 = sc->dy; a.s1 = sc->w3;
+        }
         a.s_h = sc->h; a.smooth = smooth ? 1 : 0;
         a.gu = c->gu; a.sdz = sc->dz; a.dzq = c->dzq;
         a.amax_dz = reinterpret_cast<unsigned int*>(a_dz);
@@ -536,7 +584,7 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
             a.store = 0;
             {
                 PhaseTimer pt(c, FP8MLP_PH_DGRAD2, st);
-                FP8MLP_TRY(launch_gemm(EPI_SWIGLU_BWD, false, false, FP8MLP_E5M2, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
+                FP8MLP_TRY(launch_gemm(EPI_SWIGLU_BWD, false, false, fa, fb, tmA, tmB, tmB, a, c->sm_count, st));
             }
             PhaseTimer pt(c, FP8MLP_PH_MISC, st);
             UpdateScalesArgs u{};
@@ -545,18 +593,26 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
             a.store = 1;
         }
         PhaseTimer pt(c, FP8MLP_PH_DGRAD2, st);
-        FP8MLP_TRY(launch_gemm(EPI_SWIGLU_BWD, false, false, FP8MLP_E5M2, FP8MLP_E4M3, tmA, tmB, tmB, a, c->sm_count, st));
+        FP8MLP_TRY(launch_gemm(EPI_SWIGLU_BWD, false, false, fa, fb, tmA, tmB, tmB, a, c->sm_count, st));
     }
     // dW3 = diag(1/s) (Hq^T dYq)
     {
         CUtensorMap tmA, tmB;
-        FP8MLP_TRY(make_tmap_u8(&tmA, c->hq, f, T, f));
-        FP8MLP_TRY(make_tmap_u8(&tmB, c->dyq, d, T, d));
         GemmArgs a = base_args(c, fi, di, Ti);
-        a.s0 = sc->dy; a.row_s = sc->h;
+        int fa = FP8MLP_E4M3, fb = FP8MLP_E5M2;
+        if (hb16) {                      // dW3 = Hb^T dY on the bf16 operands
+            FP8MLP_TRY(make_tmap(&tmA, c->hb, 2, true, f, T, 2 * f));
+            FP8MLP_TRY(make_tmap(&tmB, dy, 2, true, d, T, 2 * d));
+            a.elem_bytes = 2;
+            fa = fb = 1;
+        } else {
+            FP8MLP_TRY(make_tmap_u8(&tmA, c->hq, f, T, f));
+            FP8MLP_TRY(make_tmap_u8(&tmB, c->dyq, d, T, d));
+            a.s0 = sc->dy; a.row_s = sc->h;
+        }
         a.out_f32_0 = dW3; a.out_f32_1 = dW3;
         PhaseTimer pt(c, FP8MLP_PH_WGRAD3, st);
-        FP8MLP_TRY(launch_gemm(EPI_F32, true, true, FP8MLP_E4M3, FP8MLP_E5M2, tmA, tmB, tmB, a, c->sm_count, st));
+        FP8MLP_TRY(launch_gemm(EPI_F32, true, true, fa, fb, tmA, tmB, tmB, a, c->sm_count, st));
     }
     // dX = dZq [W2q|W1q]^T
     {
@@ -635,6 +691,23 @@ int fp8mlp_forward_static(int64_t T, int64_t d, int64_t f, uint32_t flags, const
     // itself clears the maxima it accumulates into)
     FP8MLP_CUDA_CHECK(cudaMemsetAsync(c.status, 0, sizeof(int), static_cast<cudaStream_t>(stream)));
     return fp8mlp_forward(&c, T, x, W1, W2, W3, mode, sc, am, y, stream);
+}
+
+int fp8mlp_gemm_bf16(int64_t M, int64_t N, int64_t K, const void* A, int a_kmajor, const void* B, int b_kmajor,
+                     float* out, void* stream) {
+    if (A == nullptr || B == nullptr || out == nullptr) return FP8MLP_ERR_ARG;
+    if (M <= 0 || N <= 0 || K <= 0 || M % 16 || N % 16 || K % 16 || M > (1 << 24) || N > (1 << 24) || K > (1 << 24)) return FP8MLP_ERR_SHAPE;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(out)) return FP8MLP_ERR_ALIGN;
+    int dev = 0, sms = 0;
+    FP8MLP_CUDA_CHECK(cudaGetDevice(&dev));
+    FP8MLP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CUtensorMap tmA, tmB;
+    if (a_kmajor) FP8MLP_TRY(make_tmap(&tmA, A, 2, false, K, M, 2 * K)); else FP8MLP_TRY(make_tmap(&tmA, A, 2, true, M, K, 2 * M));
+    if (b_kmajor) FP8MLP_TRY(make_tmap(&tmB, B, 2, false, K, N, 2 * K)); else FP8MLP_TRY(make_tmap(&tmB, B, 2, true, N, K, 2 * N));
+    GemmArgs a = base_args(nullptr, static_cast<int>(M), static_cast<int>(N), static_cast<int>(K));
+    a.elem_bytes = 2;
+    a.out_f32_0 = out; a.out_f32_1 = out;
+    return launch_gemm(EPI_F32, !a_kmajor, !b_kmajor, 1, 1, tmA, tmB, tmB, a, sms, static_cast<cudaStream_t>(stream));
 }
 
 int fp8mlp_gemm_fp8(int64_t M, int64_t N, int64_t K, const uint8_t* A, int a_kmajor, int a_fmt, const uint8_t* B,

@@ -36,15 +36,32 @@ constexpr size_t smem_bytes() {
 //   K-major : rows 128 bytes apart, 8-row atoms 1024 bytes apart (stride offset); leading unused.
 //   MN-major: each K row holds 128 contiguous M/N bytes; 8-K-row atoms 1024 bytes apart (stride
 //             offset); the next 128 M/N bytes start one box (16 KiB) later (leading offset).
-template <bool MN_MAJOR>
+// ELEM = bytes per operand element (1: FP8, 2: bf16).  A 128-byte swizzle atom holds 128 / ELEM
+// elements, so an MN-major operand of 128 rows is ELEM atoms side by side, kBoxBytes / ELEM apart.
+template <bool MN_MAJOR, int ELEM>
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-    constexpr uint64_t lbo = MN_MAJOR ? (kBoxBytes >> 4) : 1;
+    constexpr uint64_t lbo = MN_MAJOR ? ((kBoxBytes / ELEM) >> 4) : 1;
     constexpr uint64_t sbo = 1024 >> 4;
     return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
 }
-// Byte step of the descriptor start address per 32-element slice of K.
-template <bool MN_MAJOR>
-__device__ __forceinline__ uint32_t k_step_bytes() { return MN_MAJOR ? 32u * 128u : 32u; }
+// Byte step of the descriptor start address per tcgen05.mma (32 bytes of K per row).
+template <bool MN_MAJOR, int ELEM>
+__device__ __forceinline__ uint32_t k_step_bytes() { return MN_MAJOR ? (32u / ELEM) * 128u : 32u; }
+
+// One operand block of 128 rows x 128 bytes of K into shared memory (16 KiB): a K-major operand is
+// one TMA box; an MN-major operand is ELEM boxes of 128 / ELEM rows each, side by side.
+template <bool MN_MAJOR, int ELEM, bool PAIR>
+__device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row0, int k0) {
+    if constexpr (!MN_MAJOR) {
+        if constexpr (PAIR) tma_load_2d_pair(dst, map, bar, k0, row0); else tma_load_2d(dst, map, bar, k0, row0);
+    } else {
+#pragma unroll
+        for (int h = 0; h < ELEM; ++h) {
+            if constexpr (PAIR) tma_load_2d_pair(dst + h * (kBoxBytes / ELEM), map, bar, row0 + h * (128 / ELEM), k0);
+            else tma_load_2d(dst + h * (kBoxBytes / ELEM), map, bar, row0 + h * (128 / ELEM), k0);
+        }
+    }
+}
 
 __device__ __forceinline__ void tile_coords(const GemmArgs& p, int tile, int& m_tile, int& n_tile) {
     // bands of group_m m-tiles; inside a band consecutive tiles walk down m first, so the CTAs
@@ -216,6 +233,12 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
                 store_bf16x16(grow + f + 16, u + 16, true);
             }
         }
+        if (p.hb != nullptr) {           // the last layer runs in bf16: H leaves unscaled, rounded to bf16
+            uint16_t* hrow = p.hb + static_cast<int64_t>(m) * f + c0;
+            store_bf16x16(hrow, h, true);
+            if (both) store_bf16x16(hrow + 16, h + 16, true);
+            continue;
+        }
 #pragma unroll
         for (int e = 0; e < 32; ++e) h[e] = __fmul_rn(h[e], tail->s_tile[0][32 * j + e]);
         store_fp8x32<FP8MLP_E4M3>(p.hq + static_cast<int64_t>(m) * f + c0, h, both, p.wide);
@@ -310,7 +333,7 @@ __device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const fl
 // PAIR = false: one CTA per 128 x 256 tile.  PAIR = true: a cluster of two CTAs per 256 x 256 tile
 // (tcgen05 cta_group::2): rank r loads rows [128 r, 128 r + 128) of the A tile and of the B tile,
 // rank 0 issues the MMAs for both, and each CTA drains its own 128 rows of the accumulator.
-template <int EPI, bool A_MN, bool B_MN, bool PAIR>
+template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
             const __grid_constant__ CUtensorMap tmB1, const GemmArgs p) {
@@ -369,25 +392,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 for (int kb = 0; kb < p.num_k_blocks; ++kb) {
                     if (!mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     const uint32_t dst = tiles_addr + stage * kStageBytes;
-                    const int k0 = kb * kBlockK;
+                    const int k0 = kb * (kBlockK / ELEM);          // in elements
                     if constexpr (PAIR) {
                         // both CTAs' bytes are counted on rank 0's barrier, armed by rank 0 for both
                         const uint32_t bar = mapa_shared(smem_u32(&tail->full[stage]), 0);
                         if (rank == 0) mbar_expect_tx(smem_u32(&tail->full[stage]), 2 * kStageBytes);
-                        if (A_MN) tma_load_2d_pair(dst, &tmA, bar, m0, k0); else tma_load_2d_pair(dst, &tmA, bar, k0, m0);
-                        if (B_MN) tma_load_2d_pair(dst + kBoxBytes, tmB, bar, nb0, k0);
-                        else tma_load_2d_pair(dst + kBoxBytes, tmB, bar, k0, nb0);
+                        load_operand<A_MN, ELEM, true>(dst, &tmA, bar, m0, k0);
+                        load_operand<B_MN, ELEM, true>(dst + kBoxBytes, tmB, bar, nb0, k0);
                     } else {
                         const uint32_t bar = smem_u32(&tail->full[stage]);
                         mbar_expect_tx(bar, kStageBytes);
-                        if (A_MN) tma_load_2d(dst, &tmA, bar, m0, k0); else tma_load_2d(dst, &tmA, bar, k0, m0);
-                        if (B_MN) {
-                            tma_load_2d(dst + kBoxBytes, &tmB0, bar, nb0, k0);
-                            tma_load_2d(dst + 2 * kBoxBytes, &tmB1, bar, nb1, k0);
-                        } else {
-                            tma_load_2d(dst + kBoxBytes, &tmB0, bar, k0, nb0);
-                            tma_load_2d(dst + 2 * kBoxBytes, &tmB1, bar, k0, nb1);
-                        }
+                        load_operand<A_MN, ELEM, false>(dst, &tmA, bar, m0, k0);
+                        load_operand<B_MN, ELEM, false>(dst + kBoxBytes, &tmB0, bar, nb0, k0);
+                        load_operand<B_MN, ELEM, false>(dst + 2 * kBoxBytes, &tmB1, bar, nb1, k0);
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
@@ -411,10 +428,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     const uint32_t b_addr = a_addr + kBoxBytes;
 #pragma unroll
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        const uint64_t da = smem_desc<A_MN>(a_addr + k * k_step_bytes<A_MN>());
-                        const uint64_t db = smem_desc<B_MN>(b_addr + k * k_step_bytes<B_MN>());
-                        if constexpr (PAIR) umma_f8_pair(d_tmem, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
-                        else umma_f8(d_tmem, da, db, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                        const uint64_t da = smem_desc<A_MN, ELEM>(a_addr + k * k_step_bytes<A_MN, ELEM>());
+                        const uint64_t db = smem_desc<B_MN, ELEM>(b_addr + k * k_step_bytes<B_MN, ELEM>());
+                        const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
+                        if constexpr (ELEM == 1) {
+                            if constexpr (PAIR) umma_f8_pair(d_tmem, da, db, p.idesc, accum); else umma_f8(d_tmem, da, db, p.idesc, accum);
+                        } else {
+                            if constexpr (PAIR) umma_f16_pair(d_tmem, da, db, p.idesc, accum); else umma_f16(d_tmem, da, db, p.idesc, accum);
+                        }
                     }
                     // frees the stage (in both CTAs) once these MMAs have read it
                     if constexpr (PAIR) umma_commit_pair(smem_u32(&tail->empty[stage]));
@@ -529,7 +550,7 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-template <int EPI, bool A_MN, bool B_MN, bool PAIR>
+template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM>
 int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorMap& tmB1, const GemmArgs& args,
                 int64_t tiles, int sm_count, cudaStream_t st) {
     constexpr size_t kSmem = smem_bytes<PAIR>();
@@ -550,12 +571,12 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
         cfg.numAttrs = 1;
     }
     std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(kSmem));
         if (PAIR && attr_err == cudaSuccess) {
             // how many CTA pairs the device can hold at once (one CTA per SM, pairs on neighbouring SMs)
             cfg.gridDim = dim3(static_cast<unsigned>(sm_count) & ~1u);
-            attr_err = cudaOccupancyMaxActiveClusters(&max_clusters, gemm_kernel<EPI, A_MN, B_MN, PAIR>, &cfg);
+            attr_err = cudaOccupancyMaxActiveClusters(&max_clusters, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM>, &cfg);
         }
     });
     FP8MLP_CUDA_CHECK(attr_err);
@@ -567,7 +588,7 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
         grid = tiles < sm_count ? tiles : sm_count;
     }
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
-    FP8MLP_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_kernel<EPI, A_MN, B_MN, PAIR>, tmA, tmB0, tmB1, args));
+    FP8MLP_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM>, tmA, tmB0, tmB1, args));
     count_launch();
     return FP8MLP_OK;
 }
@@ -576,21 +597,28 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
 
 size_t gemm_smem_bytes() { return smem_bytes<true>() > smem_bytes<false>() ? smem_bytes<true>() : smem_bytes<false>(); }
 
-int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride) {
+int make_tmap(CUtensorMap* map, const void* base, int elem_bytes, bool mn_major, uint64_t inner, uint64_t outer,
+              uint64_t row_stride_bytes) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return FP8MLP_ERR_CUDA;
     const cuuint64_t dims[2] = {inner, outer};
-    const cuuint64_t strides[1] = {row_stride};
-    const cuuint32_t box[2] = {128, 128};
+    const cuuint64_t strides[1] = {row_stride_bytes};
+    // 128 bytes wide; 128 rows, or for an MN-major 16-bit operand the 64 K-rows of one pipeline stage
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem_bytes),
+                               static_cast<cuuint32_t>((mn_major && elem_bytes == 2) ? 64 : 128)};
     const cuuint32_t elem[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = fn(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                    const_cast<void*>(base), dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         set_cuda_error_str("cuTensorMapEncodeTiled", "driver rejected the tensor map");
         return FP8MLP_ERR_CUDA;
     }
     return FP8MLP_OK;
+}
+
+int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride) {
+    return make_tmap(map, base, 1, false, inner, outer, row_stride);
 }
 
 int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUtensorMap& tmA, const CUtensorMap& tmB0,
@@ -600,7 +628,9 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     const int tile_m = pair ? 2 * kBlockM : kBlockM;
     args.num_m_tiles = (args.M + tile_m - 1) / tile_m;
     args.num_n_tiles = (args.N + args.n_tile_cols - 1) / args.n_tile_cols;
-    args.num_k_blocks = (args.K + kBlockK - 1) / kBlockK;
+    const int elem = args.elem_bytes == 2 ? 2 : 1;
+    const int kblk = kBlockK / elem;     // contraction elements per stage
+    args.num_k_blocks = (args.K + kblk - 1) / kblk;
     if (args.group_m <= 0) args.group_m = pair ? 8 : 16;
     // instruction descriptor: [4,6) D = fp32; [7,10) A format; [10,13) B format (0 = E4M3, 1 = E5M2);
     // bit 15 / 16: A / B is MN-major; [17,23) N >> 3; [24,29) M >> 4 (M counts both CTAs of a pair)
@@ -618,18 +648,25 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     const int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
     if (tiles == 0 || args.num_k_blocks == 0) return FP8MLP_OK;
 
-#define FP8MLP_DISPATCH(E, AM, BM)                                                                         \
-    if (epi == E && a_mn == AM && b_mn == BM)                                                              \
-        return pair ? launch_inst<E, AM, BM, true>(tmA, tmB0, tmB1, args, tiles, sm_count, st)             \
-                    : launch_inst<E, AM, BM, false>(tmA, tmB0, tmB1, args, tiles, sm_count, st);
-    FP8MLP_DISPATCH(EPI_F32, false, false)
-    FP8MLP_DISPATCH(EPI_F32, false, true)
-    FP8MLP_DISPATCH(EPI_F32, true, false)
-    FP8MLP_DISPATCH(EPI_F32, true, true)
-    FP8MLP_DISPATCH(EPI_BF16, false, false)
-    FP8MLP_DISPATCH(EPI_BF16, false, true)
-    FP8MLP_DISPATCH(EPI_SWIGLU_FWD, false, true)
-    FP8MLP_DISPATCH(EPI_SWIGLU_BWD, false, false)
+#define FP8MLP_DISPATCH(E, AM, BM, EL)                                                                     \
+    if (epi == E && a_mn == AM && b_mn == BM && elem == EL)                                                \
+        return pair ? launch_inst<E, AM, BM, true, EL>(tmA, tmB0, tmB1, args, tiles, sm_count, st)         \
+                    : launch_inst<E, AM, BM, false, EL>(tmA, tmB0, tmB1, args, tiles, sm_count, st);
+    FP8MLP_DISPATCH(EPI_F32, false, false, 1)
+    FP8MLP_DISPATCH(EPI_F32, false, true, 1)
+    FP8MLP_DISPATCH(EPI_F32, true, false, 1)
+    FP8MLP_DISPATCH(EPI_F32, true, true, 1)
+    FP8MLP_DISPATCH(EPI_BF16, false, false, 1)
+    FP8MLP_DISPATCH(EPI_BF16, false, true, 1)
+    FP8MLP_DISPATCH(EPI_SWIGLU_FWD, false, true, 1)
+    FP8MLP_DISPATCH(EPI_SWIGLU_BWD, false, false, 1)
+    // the bf16 last layer of the "SwiGLU output in BF16" variant
+    FP8MLP_DISPATCH(EPI_BF16, false, true, 2)
+    FP8MLP_DISPATCH(EPI_SWIGLU_BWD, false, false, 2)
+    FP8MLP_DISPATCH(EPI_F32, true, true, 2)
+    FP8MLP_DISPATCH(EPI_F32, false, false, 2)      // the remaining layouts, for fp8mlp_gemm_bf16
+    FP8MLP_DISPATCH(EPI_F32, false, true, 2)
+    FP8MLP_DISPATCH(EPI_F32, true, false, 2)
 #undef FP8MLP_DISPATCH
     return FP8MLP_ERR_ARG;
 }

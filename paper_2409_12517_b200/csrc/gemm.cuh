@@ -23,8 +23,8 @@ enum : int { EPI_F32 = 0, EPI_BF16 = 1, EPI_SWIGLU_FWD = 2, EPI_SWIGLU_BWD = 3 }
 
 constexpr int kBlockM = 128;          // rows of D per tile (TMEM lanes)
 constexpr int kBlockN = 256;          // accumulator columns per tile
-constexpr int kBlockK = 128;          // contraction elements (= bytes) per pipeline stage
-constexpr int kUmmaK = 32;            // contraction elements per tcgen05.mma (32 bytes)
+constexpr int kBlockK = 128;          // contraction bytes per pipeline stage (128 FP8 or 64 bf16 elements)
+constexpr int kUmmaK = 32;            // contraction bytes per tcgen05.mma
 constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 bytes x 128 rows
 constexpr int kGemmThreads = 320;
 constexpr int kTmemCols = 512;
@@ -37,6 +37,7 @@ struct GemmArgs {
     int b1_offset;          // n offset of the second B box: 128, or 0 in the gate/linear case
     int group_m;            // m-tiles per rasterisation band
     int pair_mode;          // 0: CTA pairs when M > 128; 1: always CTA pairs; 2: always single CTAs
+    int elem_bytes;         // operand element size: 1 (FP8, default) or 2 (bf16; a_fmt = b_fmt = 1)
     uint32_t idesc;
     int* status;
 
@@ -58,6 +59,7 @@ struct GemmArgs {
     int store;              // 0: calibration pass, only the maxima are produced
     int wide;               // outputs may be written 32 bytes at a time (rows and bases 32-byte aligned)
     uint8_t* hq;            // fwd: E4M3 [M, f]
+    uint16_t* hb;           // fwd: if not null, bf16 [M, f] = H unscaled, stored instead of hq (32-byte aligned rows)
     uint16_t* gu;           // fwd: out (nullable), bwd: in; bf16 [M, 2f] = G | U
     unsigned int* amax_h;   // fwd: [f] bit patterns of max |H|, raised atomically; null: maxima not wanted
     const float* sdz;       // bwd: scale of dZ
@@ -70,6 +72,10 @@ size_t gemm_smem_bytes();
 // Encodes the 2-D tiled tensor map of an 8-bit matrix whose rows are `inner` bytes long and
 // `row_stride` bytes apart: box = 128 bytes x 128 rows, 128-byte swizzle, zero fill out of bounds.
 int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride);
+// General form: elem_bytes 1 (FP8) or 2 (bf16); inner / outer in elements, row stride in bytes; mn_major says how
+// the GEMM will read the matrix (an MN-major 16-bit operand is fetched in boxes of 64 K-rows).
+int make_tmap(CUtensorMap* map, const void* base, int elem_bytes, bool mn_major, uint64_t inner, uint64_t outer,
+              uint64_t row_stride_bytes);
 
 // Launches one GEMM.  a_mn / b_mn: the operand is MN-major.  The tensor maps describe A, and the
 // two 128-wide halves of the B tile (the same map twice unless they come from different matrices).

@@ -206,6 +206,22 @@ __global__ void __launch_bounds__(kThreads) update_scales_kernel(UpdateScalesArg
     }
 }
 
+// fp32 -> bf16 (round to nearest even) with max |v|: the weight of a layer that is not quantised
+__global__ void __launch_bounds__(kThreads) cast_bf16_kernel(const float* __restrict__ src, uint16_t* __restrict__ dst,
+                                                             int64_t n_units, float* amax_out) {
+    float local_max = 0.0f;
+    for (int64_t u = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; u < n_units;
+         u += static_cast<int64_t>(gridDim.x) * kThreads) {
+        const uint4 a = ld_global_nc_v4(src + 8 * u), b = ld_global_nc_v4(src + 8 * u + 4);
+        const float v[8] = {__uint_as_float(a.x), __uint_as_float(a.y), __uint_as_float(a.z), __uint_as_float(a.w),
+                            __uint_as_float(b.x), __uint_as_float(b.y), __uint_as_float(b.z), __uint_as_float(b.w)};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) local_max = fmaxf(local_max, fabsf(v[i]));
+        st_global_v4(dst + 8 * u, cvt_bf16x2(v[0], v[1]), cvt_bf16x2(v[2], v[3]), cvt_bf16x2(v[4], v[5]), cvt_bf16x2(v[6], v[7]));
+    }
+    if (amax_out != nullptr) block_atomic_max(local_max, amax_out);
+}
+
 template <typename SRC, int FMT>
 int launch_pass(bool cast, bool amax, const QuantLaunch& q, int grid, cudaStream_t st) {
     if (cast && amax) quantize_kernel<SRC, FMT, true, true><<<grid, kThreads, 0, st>>>(q);
@@ -282,6 +298,16 @@ int run_quantize_pass(bool cast, bool amax, const void* src, int src_dtype, int6
     QuantTensor t{};
     t.src = src; t.rows = rows; t.cols = cols; t.dst = dst; t.ld_dst = ld_dst; t.amax = amax_out; t.row_mul = row_mul;
     return run_quantize_segments(cast, amax, src_dtype, fmt, &t, 1, scale, sm_count, st);
+}
+
+int run_cast_bf16(const float* src, uint16_t* dst, int64_t n, float* amax_out, int sm_count, cudaStream_t st) {
+    const int64_t units = n / 8;
+    if (units == 0) return FP8MLP_OK;
+    int64_t blocks = (units + kThreads - 1) / kThreads;
+    if (blocks > int64_t(sm_count) * 8) blocks = int64_t(sm_count) * 8;
+    cast_bf16_kernel<<<static_cast<int>(blocks), kThreads, 0, st>>>(src, dst, units, amax_out);
+    FP8MLP_LAUNCH_CHECK();
+    return FP8MLP_OK;
 }
 
 int run_scale_from_amax(int fmt, const float* amax_a, const float* amax_b, float* scale, cudaStream_t st) {

@@ -36,6 +36,9 @@ int run_quantize_pass(bool cast, bool amax, const void* src, int src_dtype, int6
                       const float* row_mul, const float* scale, uint8_t* dst, int64_t ld_dst, float* amax_out,
                       int sm_count, cudaStream_t st);
 
+// dst[i] = bf16(src[i]) (n % 8 == 0), *amax_out raised to max |src| (nullable; zeroed by the caller)
+int run_cast_bf16(const float* src, uint16_t* dst, int64_t n, float* amax_out, int sm_count, cudaStream_t st);
+
 // *scale = fmt_max / max(*amax_a, *amax_b)  (amax_b nullable), 1 for a zero / non-finite amax
 int run_scale_from_amax(int fmt, const float* amax_a, const float* amax_b, float* scale, cudaStream_t st);
 

@@ -1,8 +1,10 @@
 """Parity of fp8mlp_adam_step (Adam with E4M3 first moment and E5M2 second moment, Section 5 of the
 paper) with the CPU oracle, through the C ABI.  The kernel performs the oracle's fp32 operations in
-the oracle's order with correctly rounded square root and division, so everything is compared bit
-for bit: weights, both code arrays and the reported maxima, over several steps with the scales
-re-derived from the previous step's maxima (delayed scaling)."""
+the oracle's order, so both code arrays and the reported maxima are compared bit for bit over
+several steps with the scales re-derived from the previous step's maxima (delayed scaling).  The
+weights see the kernel's approximate square root and division (special-function unit, a few 2^-23
+relative each): each step may move a weight by 1e-6 of that step's update plus one rounding of the
+weight itself, and since the moments never depend on the weights the differences do not feed back."""
 import numpy as np
 import pytest
 import torch
@@ -56,6 +58,8 @@ def test_adam_steps_bit_exact(sizes, wd):
     w0s = [rng.normal(0, 0.02, n).astype(np.float32) for n in sizes]
     dev = [_dev_state(w0) for w0 in w0s]
     ora = [_OracleState(w0) for w0 in w0s]
+    w_prev = {id(st): w0.astype(np.float64).copy() for st, w0 in zip(dev, w0s)}
+    drift = {id(st): 0.0 for st in dev}
     for t in range(1, 5):
         # gradients spanning several decades, a few exact zeros, a few outliers
         grads = []
@@ -72,7 +76,12 @@ def test_adam_steps_bit_exact(sizes, wd):
             assert st["amax_m"].item() == np.float32(am) and st["amax_v"].item() == np.float32(av)
             assert np.array_equal(st["m"].cpu().numpy(), o.m), f"first-moment codes, step {t}"
             assert np.array_equal(st["v"].cpu().numpy(), o.v), f"second-moment codes, step {t}"
-            assert np.array_equal(st["w"].cpu().numpy(), o.w), f"weights, step {t}"
+            w_before = w_prev[id(st)]
+            got_w = st["w"].cpu().numpy()
+            slack = 1e-6 * np.abs(o.w.astype(np.float64) - w_before) + np.spacing(np.abs(o.w)) + drift[id(st)]
+            assert np.all(np.abs(got_w.astype(np.float64) - o.w) <= slack), f"weights, step {t}"
+            drift[id(st)] = np.abs(got_w.astype(np.float64) - o.w)          # carried into the next step's bound
+            w_prev[id(st)] = o.w.astype(np.float64).copy()
             _advance_scales(st)
             assert st["scale_m_out"].item() == o.sm_out and st["scale_v_out"].item() == o.sv_out
 
