@@ -37,7 +37,7 @@ FP8_OVER_BF16 = 2.0          # nominal dense tensor-core ratio (4.5 vs 2.25 PFLO
 NOMINAL_FP8_TFLOPS = 4500.0
 # DRAM bytes per launch of the dominant kernel (gate/up GEMM + SwiGLU epilogue) measured by ncu
 # (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None until captured.
-NCU_TRAFFIC_BYTES = {"7b": None}
+NCU_TRAFFIC_BYTES = {"7b": 439_606_000 + 864_298_000}     # profiles/gemm_kernels_7b.txt, GEMM-1 launch
 
 
 def flops_step(T, d, f):
@@ -392,6 +392,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                 "peak_source": f"of {peak_kind}: 2 x bf16_tflops_sustained ({peaks['bf16_tflops_sustained']}) "
                                "- no FP8 GEMM peak is measured on this pool, the nominal FP8:bf16 ratio is applied",
                 "frac_of_nominal_fp8_4500": round(achieved / NOMINAL_FP8_TFLOPS, 4),
+                "algorithmic_flops_per_launch": phase_flops[dom],
+                "algorithmic_bytes_per_launch": float(T) * d + 2.0 * d * f + float(T) * f + 4.0 * T * f,
                 "step_frac_of_peak": round(value / world / fp8_peak, 4),
                 "quantize_hbm_frac": {k: v["frac_of_hbm_peak"] for k, v in kernels.items() if "gbs" in v},
                 "hbm_peak_gbs": peaks["hbm_gbs"]}

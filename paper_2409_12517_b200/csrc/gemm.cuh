@@ -1,17 +1,23 @@
-// FP8 GEMM for sm_100a: persistent, warp-specialised, tcgen05.mma kind::f8f6f4 with fp32
-// accumulators in tensor memory, operands streamed by TMA through a multi-stage shared-memory
-// ring, and the block's element-wise steps fused into the epilogue that drains tensor memory.
+// FP8 (and, for one variant, bf16) GEMM for sm_100a: persistent, warp-specialised, tcgen05.mma
+// kind::f8f6f4 / kind::f16 with fp32 accumulators in tensor memory, operands streamed by TMA through
+// a multi-stage shared-memory ring, and the block's element-wise steps fused into the epilogue that
+// drains tensor memory.
 //
 //   D[m, n] = sum_k A(m, k) * B(n, k)
 //
 // Either operand may be stored with K contiguous ("K-major", [rows, K]) or with its M/N index
-// contiguous ("MN-major", [K, rows]); both are fetched as 128-byte x 128-row TMA boxes with the
-// 128-byte swizzle and only the shared-memory matrix descriptors differ.  That lets the forward,
-// dgrad and wgrad GEMMs of the block all read the same FP8 buffers without transposed copies.
+// contiguous ("MN-major", [K, rows]); both are fetched as 128-byte-wide TMA boxes with the 128-byte
+// swizzle and only the shared-memory matrix descriptors differ.  That lets the forward, dgrad and
+// wgrad GEMMs of the block all read the same buffers without transposed copies.
+//
+// Whenever M > 128 two CTAs on neighbouring SMs (a cluster of two) share one 256 x 256 tile through
+// tcgen05 cta_group::2: each loads half of A's and half of B's rows (no multicast), the CTA of rank 0
+// issues the MMAs for both, each drains its own 128 rows of the accumulator.  Otherwise one CTA works
+// on a 128 x 256 tile.
 //
 // CTA = 10 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the MMAs,
-// warps 2-9 are the epilogue (a TMEM lane quadrant and one half of the columns each).  Two 256-column accumulators
-// alternate, so the epilogue of one tile overlaps the main loop of the next.
+// warps 2-9 are the epilogue (a TMEM lane quadrant and one half of the columns each).  Two 256-column
+// accumulators alternate, so the epilogue of one tile overlaps the main loop of the next.
 // Every wait is bounded: on expiry the CTA raises a status word and drains.
 #pragma once
 

@@ -174,3 +174,43 @@ def test_empty_batch():
         assert am["w1"].item() == oracle.amax(w.W1)
     finally:
         B.fp8mlp_destroy(ctx)
+
+
+def test_step_can_be_captured_in_a_cuda_graph_and_replays_bit_identically():
+    """Every call only enqueues kernels on the caller's stream (tensor maps travel as kernel
+    parameters, nothing allocates after fp8mlp_create), so once each kernel has run once outside a
+    capture the whole delayed-scaling step can be captured and replayed."""
+    w = wl.make_config("tiny")
+    T, d, f = w.T, w.d, w.f
+    ctx = B.fp8mlp_create(T, d, f, B.SMOOTH | B.SAVE_FOR_BWD)
+    try:
+        sc, am = B.new_scales(f), B.new_amax(f)
+        x, dy = to_dev_bf16(w.x), to_dev_bf16(w.dY)
+        W1, W2, W3 = to_dev(w.W1), to_dev(w.W2), to_dev(w.W3)
+        y = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        dx = torch.zeros_like(y)
+        dW1, dW2, dW3 = torch.zeros_like(W1), torch.zeros_like(W2), torch.zeros_like(W3)
+
+        def step(mode):
+            B.fp8mlp_forward(ctx, T, x, W1, W2, W3, mode, sc, am, y)
+            B.fp8mlp_backward(ctx, T, dy, mode, sc, am, dx, dW1, dW2, dW3)
+
+        step(B.SCALE_FROM_CURRENT_AMAX)
+        step(B.SCALE_GIVEN)
+        torch.cuda.synchronize()
+        ref = [t.clone() for t in (y, dx, dW1, dW2, dW3)]
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                step(B.SCALE_GIVEN)
+        for t in (y, dx, dW1, dW2, dW3):
+            t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert B.fp8mlp_status(ctx) == B.OK
+        for got, want in zip((y, dx, dW1, dW2, dW3), ref):
+            assert torch.equal(got.view(torch.int32) if got.dtype == torch.float32 else got.view(torch.int16),
+                               want.view(torch.int32) if want.dtype == torch.float32 else want.view(torch.int16))
+    finally:
+        B.fp8mlp_destroy(ctx)
