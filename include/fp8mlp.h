@@ -110,6 +110,12 @@ FP8MLP_API const char* fp8mlp_last_cuda_error(void);
 /* Synchronises `stream`, then returns FP8MLP_ERR_TIMEOUT if any kernel of this context gave up on
  * a bounded wait since the last call (and clears the word), else FP8MLP_OK. */
 FP8MLP_API int fp8mlp_status(fp8mlp_ctx* ctx, void* stream);
+/* Self-test of the failure path (the paper has no counterpart).  Every wait inside the kernels is bounded; this
+ * launches a one-thread kernel that waits, for at most timeout_us microseconds (1 .. 1e6), on a barrier nothing
+ * will ever complete.  The wait must give up, raise the context's status word and let the kernel end normally:
+ * returns FP8MLP_OK if it did (the next fp8mlp_status then reports FP8MLP_ERR_TIMEOUT once and clears the word,
+ * and the context stays usable), FP8MLP_ERR_STATE if the wait claimed success.  Synchronises `stream`. */
+FP8MLP_API int fp8mlp_selftest_wait_timeout(fp8mlp_ctx* ctx, int64_t timeout_us, void* stream);
 /* Device pointer and size in bytes of one of the FP8MLP_WS_* buffers (sized for T_max). */
 FP8MLP_API int fp8mlp_workspace(fp8mlp_ctx* ctx, int which, void** ptr, int64_t* bytes);
 /* Per-phase device timing (no counterpart in the paper; measurement support).  While enabled,

@@ -29,6 +29,7 @@ EXPORTS = [
     "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8", "fp8mlp_profile_enable", "fp8mlp_profile_read",
     "fp8mlp_forward_static", "fp8mlp_adam_step", "fp8mlp_scale_from_amax",
     "fp8mlp_merge_weights", "fp8mlp_forward_merged", "fp8mlp_gemm_bf16",
+    "fp8mlp_selftest_wait_timeout",
 ]
 PHASES = ["quant_x", "quant_w12", "quant_w3", "gemm1_swiglu", "gemm2_down", "quant_dy", "dgrad2_swiglu_bwd",
           "wgrad3", "dgrad1", "wgrad12", "misc"]
@@ -87,6 +88,7 @@ def lib():
         L.fp8mlp_forward_static.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_uint32, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_int, C.POINTER(_Scales), C.POINTER(_Amax),
                                             C.c_void_p, C.c_void_p]
+        L.fp8mlp_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
         L.fp8mlp_gemm_bf16.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int, C.c_void_p, C.c_int,
                                        C.c_void_p, C.c_void_p]
         L.fp8mlp_merge_weights.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
@@ -149,6 +151,11 @@ def fp8mlp_destroy(ctx: int) -> None:
 def fp8mlp_status(ctx: int) -> int:
     """Synchronises the current stream and returns OK or ERR_TIMEOUT (does not raise)."""
     return int(lib().fp8mlp_status(C.c_void_p(ctx), _stream()))
+
+
+def fp8mlp_selftest_wait_timeout(ctx: int, timeout_us: int) -> None:
+    """Runs a kernel whose bounded wait must time out; afterwards fp8mlp_status reports ERR_TIMEOUT once."""
+    _check(lib().fp8mlp_selftest_wait_timeout(C.c_void_p(ctx), timeout_us, _stream()), "fp8mlp_selftest_wait_timeout")
 
 
 def fp8mlp_workspace(ctx: int, which: int):

@@ -33,6 +33,20 @@ __global__ void zero_floats_kernel(ZeroList z) {
         z.vec[i] = 0.0f;
 }
 
+// Self-test of the bounded waits: one thread waits on a barrier that nothing ever completes, with
+// a short limit.  The wait must give up, raise the status word and let the kernel end normally.
+__global__ void wait_selftest_kernel(int* status, uint64_t timeout_ns, int* gave_up) {
+    __shared__ uint64_t never;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&never), 1);
+        abort_flag = 0;
+        mbar_init_fence();
+        const bool got = mbar_wait(smem_u32(&never), 0, &abort_flag, status, timeout_ns);
+        *gave_up = got ? 0 : 1;
+    }
+}
+
 }  // namespace fp8mlp
 
 using namespace fp8mlp;
@@ -268,6 +282,20 @@ int fp8mlp_status(fp8mlp_ctx* c, void* stream) {
         return FP8MLP_ERR_TIMEOUT;
     }
     return FP8MLP_OK;
+}
+
+int fp8mlp_selftest_wait_timeout(fp8mlp_ctx* c, int64_t timeout_us, void* stream) {
+    if (c == nullptr) return FP8MLP_ERR_ARG;
+    if (timeout_us < 1 || timeout_us > 1000000) return FP8MLP_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* gave_up = reinterpret_cast<int*>(c->dummy + 6);      // a spare word of the context
+    FP8MLP_CUDA_CHECK(cudaMemsetAsync(gave_up, 0, sizeof(int), st));
+    wait_selftest_kernel<<<1, 32, 0, st>>>(c->status, static_cast<uint64_t>(timeout_us) * 1000ull, gave_up);
+    FP8MLP_LAUNCH_CHECK();
+    int flag = 0;
+    FP8MLP_CUDA_CHECK(cudaMemcpyAsync(&flag, gave_up, sizeof(int), cudaMemcpyDeviceToHost, st));
+    FP8MLP_CUDA_CHECK(cudaStreamSynchronize(st));
+    return flag == 1 ? FP8MLP_OK : FP8MLP_ERR_STATE;
 }
 
 int fp8mlp_profile_enable(fp8mlp_ctx* c, int on) {

@@ -127,14 +127,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false if the CTA is aborting or the wait ran out of time, in which case
 // it raises the CTA's abort flag (shared) and the global status word; the caller leaves its loop.
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // 2 s: far beyond any kernel of this library
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort, int* status,
+                                          uint64_t timeout_ns = kWaitTimeoutNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 63u) == 0u) {
             if (*cta_abort) return false;
-            if (global_timer_ns() - t0 > kWaitTimeoutNs) {
+            if (global_timer_ns() - t0 > timeout_ns) {
                 *cta_abort = 1;
                 if (status != nullptr) atomicExch(status, STATUS_WAIT_TIMEOUT);
                 return false;
