@@ -80,6 +80,33 @@ __device__ __forceinline__ float warp_max_nonneg(float v) {
     return __uint_as_float(r);
 }
 
+// Two fp32 values in one 64-bit register, operated on by one instruction (sm_100).  Each half is
+// rounded exactly like the scalar operation, so results do not change - only the instruction count.
+typedef uint64_t f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 // sigma(z) = 1 / (1 + e^-z) in fp32 on the special-function unit: 2^x and 1/x to about 2^-22
 // relative, which moves a later FP8 code by one step only where the exact value sits that close
 // to a rounding boundary.  e^-z overflowing to +inf gives 0, underflowing gives 1.

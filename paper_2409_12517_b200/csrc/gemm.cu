@@ -278,6 +278,11 @@ __device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const fl
     const int f = p.N;
     float local_max = 0.0f;
     GuChunk next;
+    // A power-of-two sdz (what fp8mlp_update_scales produces) commutes with every rounding below, so it
+    // is folded into the dequantisation factor: dG, dU come out already scaled, bit for bit the same as
+    // scaling them at the end, and the running maximum is scaled back once.
+    const bool fold = (__float_as_uint(sdz) & 0x007FFFFFu) == 0u && sdz > 1.0e-30f && sdz < 1.0e30f;
+    if (fold) dq = __fmul_rn(dq, sdz);
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj) {
         GuChunk& cur = (jj & 1) ? next : first;
@@ -289,44 +294,54 @@ __device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const fl
         tmem_ld32(taddr + 32 * j, acc);
         if (jj < 3) load_gu(p, m, c0 + 32, nxt);
         tmem_ld_wait();
+        // element pairs (2q, 2q+1) travel as one 64-bit register through the multiplies and adds
         float dg[32], du[32];
+        f32x2 dh2[16], g2[16], sig2[16];
+        const f32x2 dq2 = pack2(dq, dq), one2 = pack2(1.0f, 1.0f), nl2 = pack2(-1.4426950408889634f, -1.4426950408889634f);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            float dh = __fmul_rn(__uint_as_float(acc[e]), dq);
-            if (p.smooth) dh = __fmul_rn(dh, s_tile[32 * j + e]);
-            du[e] = dh;
+        for (int q = 0; q < 16; ++q) {
+            dh2[q] = mul2(pack2(__uint_as_float(acc[2 * q]), __uint_as_float(acc[2 * q + 1])), dq2);
+            if (p.smooth) dh2[q] = mul2(dh2[q], pack2(s_tile[32 * j + 2 * q], s_tile[32 * j + 2 * q + 1]));
+            g2[q] = pack2(bf16_lo(cur.g[q]), bf16_hi(cur.g[q]));
         }
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            const uint32_t gw = cur.g[e >> 1];
-            const float g = (e & 1) ? bf16_hi(gw) : bf16_lo(gw);
-            dg[e] = ex2_approx(__fmul_rn(g, -1.4426950408889634f));
+        for (int q = 0; q < 16; ++q) {
+            float a, b;
+            unpack2(mul2(g2[q], nl2), a, b);
+            sig2[q] = pack2(ex2_approx(a), ex2_approx(b));
         }
 #pragma unroll
-        for (int e = 0; e < 32; ++e) dg[e] = rcp_approx(__fadd_rn(1.0f, dg[e]));         // sigma(G)
+        for (int q = 0; q < 16; ++q) {
+            float a, b;
+            unpack2(add2(one2, sig2[q]), a, b);
+            sig2[q] = pack2(rcp_approx(a), rcp_approx(b));                                  // sigma(G)
+        }
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            const uint32_t gw = cur.g[e >> 1], uw = cur.u[e >> 1];
-            const float g = (e & 1) ? bf16_hi(gw) : bf16_lo(gw);
-            const float u = (e & 1) ? bf16_hi(uw) : bf16_lo(uw);
-            const float dh = du[e], sig = dg[e];
-            du[e] = __fmul_rn(dh, __fmul_rn(g, sig));
-            const float t1 = __fadd_rn(1.0f, __fmul_rn(g, __fsub_rn(1.0f, sig)));
-            dg[e] = __fmul_rn(__fmul_rn(dh, u), __fmul_rn(sig, t1));
-            local_max = fmaxf(local_max, fmaxf(fabsf(dg[e]), fabsf(du[e])));
+        for (int q = 0; q < 16; ++q) {
+            const f32x2 u2 = pack2(bf16_lo(cur.u[q]), bf16_hi(cur.u[q]));
+            const f32x2 du_2 = mul2(dh2[q], mul2(g2[q], sig2[q]));
+            const f32x2 t1 = add2(one2, mul2(g2[q], sub2(one2, sig2[q])));
+            const f32x2 dg_2 = mul2(mul2(dh2[q], u2), mul2(sig2[q], t1));
+            unpack2(du_2, du[2 * q], du[2 * q + 1]);
+            unpack2(dg_2, dg[2 * q], dg[2 * q + 1]);
+            local_max = fmaxf(local_max, fmaxf(fmaxf(fabsf(dg[2 * q]), fabsf(dg[2 * q + 1])),
+                                               fmaxf(fabsf(du[2 * q]), fabsf(du[2 * q + 1]))));
         }
         if (!p.store || !row_ok) continue;
+        if (!fold) {
+            const f32x2 sdz2 = pack2(sdz, sdz);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            dg[e] = __fmul_rn(dg[e], sdz);
-            du[e] = __fmul_rn(du[e], sdz);
+            for (int q = 0; q < 16; ++q) {
+                unpack2(mul2(pack2(dg[2 * q], dg[2 * q + 1]), sdz2), dg[2 * q], dg[2 * q + 1]);
+                unpack2(mul2(pack2(du[2 * q], du[2 * q + 1]), sdz2), du[2 * q], du[2 * q + 1]);
+            }
         }
         uint8_t* zrow = p.dzq + static_cast<int64_t>(m) * 2 * f + c0;
         const bool both = c0 + 16 < f;
         store_fp8x32<FP8MLP_E5M2>(zrow, dg, both, p.wide);
         store_fp8x32<FP8MLP_E5M2>(zrow + f, du, both, p.wide);
     }
-    return local_max;
+    return fold ? __fmul_rn(local_max, __fdiv_rn(1.0f, sdz)) : local_max;
 }
 
 // ---------------------------------------------------------------- the kernel
