@@ -10,9 +10,17 @@ namespace {
 // ---------------------------------------------------------------- shared memory plan
 // Single CTA: a stage holds an A box and two B boxes (128 x 256 tile).  CTA pair: a stage holds this
 // CTA's A box and its one B box (its halves of a 256 x 256 tile).
-template <bool PAIR> struct Plan;
-template <> struct Plan<false> { static constexpr int kStages = 4, kStageBytes = 3 * kBoxBytes, kTileM = 128; };
-template <> struct Plan<true>  { static constexpr int kStages = 6, kStageBytes = 2 * kBoxBytes, kTileM = 256; };
+// The backward SwiGLU kernel gives up stages for a ring of two 32-KiB slots through which a loader
+// warp streams the saved G and U (a 128-row x 64-channel bf16 box each) to the epilogue.
+constexpr int kGuSlots = 2;
+constexpr int kGuSlotBytes = 2 * kBoxBytes;
+template <bool PAIR, int EPI> struct Plan;
+template <int EPI> struct Plan<false, EPI> {
+    static constexpr int kStages = EPI == EPI_SWIGLU_BWD ? 3 : 4, kStageBytes = 3 * kBoxBytes, kTileM = 128;
+};
+template <int EPI> struct Plan<true, EPI> {
+    static constexpr int kStages = EPI == EPI_SWIGLU_BWD ? 4 : 6, kStageBytes = 2 * kBoxBytes, kTileM = 256;
+};
 constexpr int kMaxStages = 6;
 
 struct __align__(8) SmemTail {
@@ -20,14 +28,17 @@ struct __align__(8) SmemTail {
     uint64_t empty[kMaxStages];  // MMA -> TMA: stage drained
     uint64_t tmem_full[2];       // MMA -> epilogue: accumulator complete
     uint64_t tmem_empty[2];      // epilogue -> MMA: accumulator drained (CTA pair: rank 0's count both CTAs)
+    uint64_t gu_full[kGuSlots];  // loader -> epilogue: saved G, U chunk landed (backward)
+    uint64_t gu_empty[kGuSlots]; // epilogue -> loader: chunk read into registers
     uint32_t tmem_base;
     int abort;
     float s_tile[2][kBlockN];    // per-channel scales of the current tile(s)
     unsigned int amax_tile[128]; // per-channel maxima of the current tile (forward)
 };
-template <bool PAIR>
+template <bool PAIR, int EPI>
 constexpr size_t smem_bytes() {
-    return 1024 /*alignment slack*/ + size_t(Plan<PAIR>::kStages) * Plan<PAIR>::kStageBytes + sizeof(SmemTail);
+    return 1024 /*alignment slack*/ + size_t(Plan<PAIR, EPI>::kStages) * Plan<PAIR, EPI>::kStageBytes +
+           (EPI == EPI_SWIGLU_BWD ? size_t(kGuSlots) * kGuSlotBytes : 0) + sizeof(SmemTail);
 }
 
 // ---------------------------------------------------------------- descriptors
@@ -245,55 +256,49 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
     }
 }
 
-// Saved bf16 G and U of one row, 32 channels each (4 x 32 bytes), for the backward epilogue.
-struct GuChunk { uint32_t g[16], u[16]; };
-__device__ __forceinline__ void load_gu(const GemmArgs& p, int m, int c0, GuChunk& r) {
-    const int f = p.N;
-    const bool lo = m < p.M && c0 < f, hi = m < p.M && c0 + 16 < f;
-    const uint16_t* grow = p.gu + static_cast<int64_t>(m) * 2 * f + c0;
-    uint32_t(&g0)[8] = *reinterpret_cast<uint32_t(*)[8]>(r.g);
-    uint32_t(&g1)[8] = *reinterpret_cast<uint32_t(*)[8]>(r.g + 8);
-    uint32_t(&u0)[8] = *reinterpret_cast<uint32_t(*)[8]>(r.u);
-    uint32_t(&u1)[8] = *reinterpret_cast<uint32_t(*)[8]>(r.u + 8);
-    if (lo) { ld_global_nc_v8(grow, g0); ld_global_nc_v8(grow + f, u0); }
-    else {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) { g0[e] = 0u; u0[e] = 0u; }
-    }
-    if (hi) { ld_global_nc_v8(grow + 16, g1); ld_global_nc_v8(grow + f + 16, u1); }
-    else {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) { g1[e] = 0u; u1[e] = 0u; }
-    }
-}
-
-// Backward: accumulator = dY W3'^T for 256 channels; this warp takes [128 half, 128 half + 128).
+// Backward: accumulator = dY W3'^T for 256 channels, worked through in four chunks of 64 channels; of
+// each chunk this warp takes channels [32 half, 32 half + 32).  The saved bf16 G and U of a chunk arrive
+// in shared memory (loader warp, TMA, 128-byte swizzle: the 16-byte piece j of row r sits at piece
+// j ^ (r & 7)); the thread copies its row's 64 + 64 bytes to registers and hands the slot back.
 // dH = acc * dq (* s_i with Smooth-SwiGLU); dU = dH * G sigma(G);
 // dG = dH * U * sigma(G) (1 + G (1 - sigma(G))); max of |dG|, |dU|; dZq = Q_e5m2([dG | dU] * sdz).
-// `first` holds the saved G, U of the first chunk, requested before the accumulator was ready;
-// each chunk requests the next one's before it starts computing.
-__device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const float* s_tile, uint32_t taddr, int half,
-                                                     int m, int n0, float dq, float sdz, GuChunk& first) {
+// Returns false if a wait ran out.
+__device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail* tail, uint32_t gu_base, uint32_t& gu_count,
+                                                    const float* s_tile, uint32_t taddr, int lane, int half, int row,
+                                                    int m, int n0, float dq, float sdz, volatile int* abort_flag,
+                                                    float& run_max) {
     const bool row_ok = m < p.M;
     const int f = p.N;
     float local_max = 0.0f;
-    GuChunk next;
     // A power-of-two sdz (what fp8mlp_update_scales produces) commutes with every rounding below, so it
     // is folded into the dequantisation factor: dG, dU come out already scaled, bit for bit the same as
     // scaling them at the end, and the running maximum is scaled back once.
     const bool fold = (__float_as_uint(sdz) & 0x007FFFFFu) == 0u && sdz > 1.0e-30f && sdz < 1.0e30f;
     if (fold) dq = __fmul_rn(dq, sdz);
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c, ++gu_count) {
+        const uint32_t slot = gu_count % kGuSlots, phase = (gu_count / kGuSlots) & 1u;
+        const int col = 64 * c + 32 * half;            // first of this warp's 32 accumulator columns
+        const int c0 = n0 + col;
+        if (!mbar_wait(smem_u32(&tail->gu_full[slot]), phase, abort_flag, p.status)) return false;
+        uint4 gq[4], uq[4];
+        {
+            const uint32_t rbase = gu_base + slot * kGuSlotBytes + static_cast<uint32_t>(row) * 128u;
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-        GuChunk& cur = (jj & 1) ? next : first;
-        GuChunk& nxt = (jj & 1) ? first : next;
-        const int j = 4 * half + jj;
-        const int c0 = n0 + 32 * j;
-        if (c0 >= f) break;
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t off = static_cast<uint32_t>(((4 * half + i) ^ (row & 7)) * 16);
+                gq[i] = ld_shared_v4(rbase + off);
+                uq[i] = ld_shared_v4(rbase + kBoxBytes + off);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tail->gu_empty[slot]));     // the chunk is in registers
+        if (c0 >= f) continue;
         uint32_t acc[32];
-        tmem_ld32(taddr + 32 * j, acc);
-        if (jj < 3) load_gu(p, m, c0 + 32, nxt);
+        tmem_ld32(taddr + col, acc);
         tmem_ld_wait();
+        const uint32_t* gw = reinterpret_cast<const uint32_t*>(gq);
+        const uint32_t* uw = reinterpret_cast<const uint32_t*>(uq);
         // element pairs (2q, 2q+1) travel as one 64-bit register through the multiplies and adds
         float dg[32], du[32];
         f32x2 dh2[16], g2[16], sig2[16];
@@ -301,8 +306,8 @@ __device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const fl
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             dh2[q] = mul2(pack2(__uint_as_float(acc[2 * q]), __uint_as_float(acc[2 * q + 1])), dq2);
-            if (p.smooth) dh2[q] = mul2(dh2[q], pack2(s_tile[32 * j + 2 * q], s_tile[32 * j + 2 * q + 1]));
-            g2[q] = pack2(bf16_lo(cur.g[q]), bf16_hi(cur.g[q]));
+            if (p.smooth) dh2[q] = mul2(dh2[q], pack2(s_tile[col + 2 * q], s_tile[col + 2 * q + 1]));
+            g2[q] = pack2(bf16_lo(gw[q]), bf16_hi(gw[q]));
         }
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
@@ -318,7 +323,7 @@ __device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const fl
         }
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
-            const f32x2 u2 = pack2(bf16_lo(cur.u[q]), bf16_hi(cur.u[q]));
+            const f32x2 u2 = pack2(bf16_lo(uw[q]), bf16_hi(uw[q]));
             const f32x2 du_2 = mul2(dh2[q], mul2(g2[q], sig2[q]));
             const f32x2 t1 = add2(one2, mul2(g2[q], sub2(one2, sig2[q])));
             const f32x2 dg_2 = mul2(mul2(dh2[q], u2), mul2(sig2[q], t1));
@@ -341,7 +346,8 @@ __device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const fl
         store_fp8x32<FP8MLP_E5M2>(zrow, dg, both, p.wide);
         store_fp8x32<FP8MLP_E5M2>(zrow + f, du, both, p.wide);
     }
-    return fold ? __fmul_rn(local_max, __fdiv_rn(1.0f, sdz)) : local_max;
+    run_max = fmaxf(run_max, fold ? __fmul_rn(local_max, __fdiv_rn(1.0f, sdz)) : local_max);
+    return true;
 }
 
 // ---------------------------------------------------------------- the kernel
@@ -351,14 +357,18 @@ __device__ __forceinline__ float epilogue_swiglu_bwd(const GemmArgs& p, const fl
 template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
-            const __grid_constant__ CUtensorMap tmB1, const GemmArgs p) {
-    constexpr int kStages = Plan<PAIR>::kStages;
-    constexpr int kStageBytes = Plan<PAIR>::kStageBytes;
+            const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmG,
+            const __grid_constant__ CUtensorMap tmU, const GemmArgs p) {
+    constexpr int kStages = Plan<PAIR, EPI>::kStages;
+    constexpr int kStageBytes = Plan<PAIR, EPI>::kStageBytes;
+    constexpr int kTileM = Plan<PAIR, EPI>::kTileM;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;         // swizzle atoms need 1024-byte alignment
     uint8_t* tiles_ptr = smem_raw + (tiles_addr - raw_addr);
-    SmemTail* tail = reinterpret_cast<SmemTail*>(tiles_ptr + size_t(kStages) * kStageBytes);
+    constexpr uint32_t kRingBytes = EPI == EPI_SWIGLU_BWD ? kGuSlots * kGuSlotBytes : 0;
+    const uint32_t gu_base = tiles_addr + kStages * kStageBytes;     // ring of saved G, U chunks (backward only)
+    SmemTail* tail = reinterpret_cast<SmemTail*>(tiles_ptr + size_t(kStages) * kStageBytes + kRingBytes);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -375,6 +385,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&tail->full[s]), 1);
             mbar_init(smem_u32(&tail->empty[s]), 1);
+        }
+        for (int b = 0; b < kGuSlots; ++b) {
+            mbar_init(smem_u32(&tail->gu_full[b]), 1);
+            mbar_init(smem_u32(&tail->gu_empty[b]), kEpiThreads / 32);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&tail->tmem_full[b]), 1);
@@ -401,7 +415,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
                 int m_tile, n_tile;
                 tile_coords(p, tile, m_tile, n_tile);
-                const int m0 = m_tile * Plan<PAIR>::kTileM + static_cast<int>(rank) * kBlockM;
+                const int m0 = m_tile * kTileM + static_cast<int>(rank) * kBlockM;
                 const int nb0 = n_tile * p.n_tile_cols + (PAIR ? static_cast<int>(rank) * p.b1_offset : 0);
                 const int nb1 = nb0 + p.b1_offset;
                 for (int kb = 0; kb < p.num_k_blocks; ++kb) {
@@ -463,6 +477,31 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
             }
         }
+    } else if (warp == 10) {
+        // ------------------------------------------------------------ loader of the saved G, U (backward only)
+        if constexpr (EPI == EPI_SWIGLU_BWD) {
+            if (lane == 0) {
+                tma_prefetch_desc(&tmG);
+                tma_prefetch_desc(&tmU);
+                uint32_t count = 0;
+                bool ok = true;
+                for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
+                    int m_tile, n_tile;
+                    tile_coords(p, tile, m_tile, n_tile);
+                    const int m0 = m_tile * kTileM + static_cast<int>(rank) * kBlockM;
+                    const int n0 = n_tile * p.n_tile_cols;
+                    for (int c = 0; c < 4; ++c, ++count) {
+                        const uint32_t slot = count % kGuSlots, phase = (count / kGuSlots) & 1u;
+                        if (!mbar_wait(smem_u32(&tail->gu_empty[slot]), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                        const uint32_t bar = smem_u32(&tail->gu_full[slot]);
+                        const uint32_t dst = gu_base + slot * kGuSlotBytes;
+                        mbar_expect_tx(bar, kGuSlotBytes);
+                        tma_load_2d(dst, &tmG, bar, n0 + 64 * c, m0);              // columns past f read as zeros
+                        tma_load_2d(dst + kBoxBytes, &tmU, bar, n0 + 64 * c, m0);
+                    }
+                }
+            }
+        }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..9)
         const int quad = warp & 3;                     // TMEM lanes [32*quad, 32*quad+32) belong to this warp
@@ -473,11 +512,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         float sdz = 1.0f;
         if constexpr (EPI == EPI_SWIGLU_BWD) sdz = *p.sdz;
         float run_max = 0.0f;
+        uint32_t gu_count = 0;                         // chunks of saved G, U consumed so far (backward)
         int it = 0;
         for (int tile = first_tile; tile < num_tiles; tile += tile_step, ++it) {
             int m_tile, n_tile;
             tile_coords(p, tile, m_tile, n_tile);
-            const int m = m_tile * Plan<PAIR>::kTileM + static_cast<int>(rank) * kBlockM + row;
+            const int m = m_tile * kTileM + static_cast<int>(rank) * kBlockM + row;
             const int n0 = n_tile * p.n_tile_cols;
             const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
             if constexpr (EPI == EPI_SWIGLU_FWD) {
@@ -486,11 +526,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     tail->amax_tile[et] = 0u;
                 }
             }
-            GuChunk gu_first;
-            if constexpr (EPI == EPI_SWIGLU_BWD) {
-                tail->s_tile[acc][et] = (n0 + et) < p.N ? p.s_h[n0 + et] : 1.0f;
-                load_gu(p, m, n0 + 128 * half, gu_first);   // does not depend on the accumulator
-            }
+            if constexpr (EPI == EPI_SWIGLU_BWD) tail->s_tile[acc][et] = (n0 + et) < p.N ? p.s_h[n0 + et] : 1.0f;
             const bool got = mbar_wait(smem_u32(&tail->tmem_full[acc]), acc_phase, abort_flag, p.status);
             if (!epi_all(got)) break;                  // also orders the s_tile / amax_tile writes above
             tc_fence_after();
@@ -505,7 +541,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
                 epilogue_swiglu_fwd(p, tail, taddr, lane, half, m, n0, dq0);
             } else {
-                run_max = fmaxf(run_max, epilogue_swiglu_bwd(p, tail->s_tile[acc], taddr, half, m, n0, dq0, sdz, gu_first));
+                const bool fine = epilogue_swiglu_bwd(p, tail, gu_base, gu_count, tail->s_tile[acc], taddr, lane, half, row,
+                                                      m, n0, dq0, sdz, abort_flag, run_max);
+                if (!epi_all(fine)) break;
             }
             // accumulator drained: hand it back to the MMA warp (of rank 0)
             tc_fence_before();
@@ -568,7 +606,15 @@ EncodeTiledFn encode_fn() {
 template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM>
 int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorMap& tmB1, const GemmArgs& args,
                 int64_t tiles, int sm_count, cudaStream_t st) {
-    constexpr size_t kSmem = smem_bytes<PAIR>();
+    constexpr size_t kSmem = smem_bytes<PAIR, EPI>();
+    // the saved activations [M, 2f] bf16 as two matrices of f columns: G, and U starting f elements in
+    CUtensorMap tmG = tmA, tmU = tmA;
+    if (EPI == EPI_SWIGLU_BWD) {
+        const uint64_t f = static_cast<uint64_t>(args.N), rows = static_cast<uint64_t>(args.M);
+        int rc = make_tmap(&tmG, args.gu, 2, false, f, rows, 4 * f);
+        if (rc == FP8MLP_OK) rc = make_tmap(&tmU, args.gu + f, 2, false, f, rows, 4 * f);
+        if (rc != FP8MLP_OK) return rc;
+    }
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     static int max_clusters = 0;
@@ -603,14 +649,14 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
         grid = tiles < sm_count ? tiles : sm_count;
     }
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
-    FP8MLP_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM>, tmA, tmB0, tmB1, args));
+    FP8MLP_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM>, tmA, tmB0, tmB1, tmG, tmU, args));
     count_launch();
     return FP8MLP_OK;
 }
 
 }  // namespace
 
-size_t gemm_smem_bytes() { return smem_bytes<true>() > smem_bytes<false>() ? smem_bytes<true>() : smem_bytes<false>(); }
+size_t gemm_smem_bytes() { return smem_bytes<true, EPI_F32>(); }
 
 int make_tmap(CUtensorMap* map, const void* base, int elem_bytes, bool mn_major, uint64_t inner, uint64_t outer,
               uint64_t row_stride_bytes) {

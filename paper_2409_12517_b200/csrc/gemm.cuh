@@ -15,8 +15,9 @@
 // issues the MMAs for both, each drains its own 128 rows of the accumulator.  Otherwise one CTA works
 // on a 128 x 256 tile.
 //
-// CTA = 10 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the MMAs,
-// warps 2-9 are the epilogue (a TMEM lane quadrant and one half of the columns each).  Two 256-column
+// CTA = 11 warps: warp 0 issues TMA loads, warp 1 owns tensor memory and issues the MMAs,
+// warps 2-9 are the epilogue (a TMEM lane quadrant and one half of the columns each), warp 10
+// streams the saved G, U to the backward SwiGLU epilogue (idle elsewhere).  Two 256-column
 // accumulators alternate, so the epilogue of one tile overlaps the main loop of the next.
 // Every wait is bounded: on expiry the CTA raises a status word and drains.
 #pragma once
@@ -32,7 +33,7 @@ constexpr int kBlockN = 256;          // accumulator columns per tile
 constexpr int kBlockK = 128;          // contraction bytes per pipeline stage (128 FP8 or 64 bf16 elements)
 constexpr int kUmmaK = 32;            // contraction bytes per tcgen05.mma
 constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 bytes x 128 rows
-constexpr int kGemmThreads = 320;
+constexpr int kGemmThreads = 352;       // TMA warp, MMA warp, 8 epilogue warps, loader warp of the saved activations
 constexpr int kTmemCols = 512;
 constexpr int kEpiThreads = 256;
 
@@ -85,6 +86,7 @@ int make_tmap(CUtensorMap* map, const void* base, int elem_bytes, bool mn_major,
 
 // Launches one GEMM.  a_mn / b_mn: the operand is MN-major.  The tensor maps describe A, and the
 // two 128-wide halves of the B tile (the same map twice unless they come from different matrices).
+// EPI_SWIGLU_BWD reads args.gu through TMA: the launcher builds those two tensor maps itself.
 int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUtensorMap& tmA,
                 const CUtensorMap& tmB0, const CUtensorMap& tmB1, GemmArgs args, int sm_count, cudaStream_t st);
 
