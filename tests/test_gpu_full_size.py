@@ -234,3 +234,41 @@ def test_7b_forward_smooth_on_versus_off_code_statistics():
     typical = np.delete(off["chan_top"], out_ch)
     assert np.median(typical) <= 0x76 - 3 * 8                            # three binades or more below the top
     assert off["zero_frac"] > 3 * on["zero_frac"]
+
+
+def test_7b_forward_just_in_time_scales_sampled_channels():
+    """The forward-only 7B configuration in the mode it is stated in (every scale from the current
+    data, Smooth-SwiGLU on), at full size: the per-tensor scales of x and [W2|W1] against the
+    oracle's maxima of the whole tensors, and for a sample of channels (all outlier channels among
+    them) the per-channel maxima over all 4096 tokens, the s_i derived from them and the resulting
+    code columns - a channel's maximum, scale and codes depend on no other channel."""
+    w = wl.make_config("7b_fwd")
+    T, d, f = w.T, w.d, w.f
+    rng = np.random.default_rng(77)
+    chans = _sample(rng, f, 40, w.outlier_channels)
+    ctx = B.fp8mlp_create(T, d, f, B.SMOOTH)
+    try:
+        sc, am = B.new_scales(f), B.new_amax(f)
+        y = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        B.fp8mlp_forward(ctx, T, to_dev_bf16(w.x), to_dev(w.W1), to_dev(w.W2), to_dev(w.W3), B.SCALE_FROM_CURRENT_AMAX, sc, am, y)
+        assert B.fp8mlp_status(ctx) == B.OK
+        ci = torch.from_numpy(chans).cuda()
+        hq_cols = B.workspace_tensor(ctx, B.WS_HQ, (T, f), torch.uint8)[:, ci].cpu().numpy()
+        scales = {k: v.cpu().numpy() for k, v in sc.items()}
+        amax = {k: v.cpu().numpy() for k, v in am.items()}
+    finally:
+        B.fp8mlp_destroy(ctx)
+    a_x = oracle.amax(wl.bf16_bits_to_f32(w.x))
+    a_w = max(oracle.amax(w.W1), oracle.amax(w.W2))
+    sx, sw12 = oracle.scale_from_amax(oracle.E4M3, a_x), oracle.scale_from_amax(oracle.E4M3, a_w)
+    assert amax["x"][0] == np.float32(a_x) and scales["x"][0] == np.float32(sx) and scales["w12"][0] == np.float32(sw12)
+    # the channel sub-problem with those two scales given: its per-channel maxima are the full run's
+    probe = oracle.forward(w.x, w.W1[:, chans], w.W2[:, chans], w.W3[chans, :], scale_mode=oracle.SCALE_GIVEN,
+                           sx=sx, sw12=sw12, s_h=np.ones(chans.size, np.float32), sw3=1.0)
+    assert np.allclose(amax["h"][chans], probe["amax_h"], rtol=AMAX_RTOL, atol=0)
+    s_ref = np.array([oracle.pow2_scale(oracle.E4M3, a) for a in probe["amax_h"]], np.float32)
+    assert np.array_equal(scales["h"][chans], s_ref), "s_i of the sampled channels"
+    fwc = oracle.forward(w.x, w.W1[:, chans], w.W2[:, chans], w.W3[chans, :], scale_mode=oracle.SCALE_GIVEN,
+                         sx=sx, sw12=sw12, s_h=s_ref, sw3=1.0)
+    frac, worst = code_mismatch(hq_cols, fwc["Hq"])
+    assert worst <= 1 and frac <= CODE_FRAC, f"Hq columns: {frac:.2e} differ, worst {worst}"
