@@ -314,6 +314,21 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         adam = {"ms": round(adam_ms, 4), "params": 3 * d * f, "bytes_per_param": 16,
                 "gbs": round(adam_bytes / (adam_ms * 1e-3) / 1e9, 1)}
         del states
+    # the same step with every scale derived just in time (extra amax passes, GEMM-1 and dgrad-2 run twice)
+    jit = None
+    if rank == 0:
+        for _ in range(2):
+            step(B.SCALE_FROM_CURRENT_AMAX)
+        torch.cuda.synchronize()
+        n_jit = max(1, min(args.steps, 20))
+        e0.record()
+        for _ in range(n_jit):
+            step(B.SCALE_FROM_CURRENT_AMAX)
+        e1.record()
+        torch.cuda.synchronize()
+        jit_ms = e0.elapsed_time(e1) / n_jit
+        jit = {"ms_per_step": round(jit_ms, 4), "tflops_useful": round(job_tflops(T, d, f, 1, jit_ms), 1)}
+        step(B.SCALE_GIVEN)
     # inference form (s folded into the weights once; not part of the metric): forward only, weights static
     merged = None
     if rank == 0:
@@ -419,6 +434,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         adam["frac_of_hbm_peak"] = round(adam["gbs"] / peaks["hbm_gbs"], 3)
         merged["frac_of_fp8_peak"] = round(merged["tflops"] / fp8_peak, 3)
         out["beside_the_step"] = {"adam_fp8_moments": adam, "inference_merged_forward": merged,
+                                  "step_with_just_in_time_scales": jit,
                                   "step_with_smooth_swiglu_off": plain,
                                   "step_with_swiglu_output_in_bf16": hbf16,
                                   "note": "Adam with E4M3/E5M2 moments on W1, W2, W3, and the inference form of "
