@@ -214,3 +214,32 @@ def test_step_can_be_captured_in_a_cuda_graph_and_replays_bit_identically():
                                want.view(torch.int32) if want.dtype == torch.float32 else want.view(torch.int16))
     finally:
         B.fp8mlp_destroy(ctx)
+
+
+def test_empty_inputs_of_the_other_entry_points():
+    """T = 0 and n = 0 are legal everywhere: nothing is launched on data, maxima read zero."""
+    ctx = B.fp8mlp_create(16, 64, 64, B.SMOOTH)
+    hb = B.fp8mlp_create(16, 64, 64, B.H_BF16 | B.SAVE_FOR_BWD)
+    try:
+        w = wl.make("e2", 3, 16, 64, 64, w_std=0.05)
+        sc, am = B.new_scales(64), B.new_amax(64)
+        W1, W2, W3 = to_dev(w.W1), to_dev(w.W2), to_dev(w.W3)
+        s = torch.ones(64, device="cuda")
+        B.fp8mlp_merge_weights(ctx, W1, W2, W3, s, B.SCALE_FROM_CURRENT_AMAX, sc, am)
+        B.fp8mlp_forward_merged(ctx, 0, None, B.SCALE_GIVEN, sc, None, None)
+        B.fp8mlp_forward(hb, 0, None, W1, W2, W3, B.SCALE_FROM_CURRENT_AMAX, sc, am, None)
+        g = [torch.full((64, 64), 3.0, device="cuda") for _ in range(3)]
+        B.fp8mlp_backward(hb, 0, None, B.SCALE_FROM_CURRENT_AMAX, sc, am, None, g[0], g[1], g[2])
+        one = lambda: torch.ones(1, device="cuda")
+        empty = dict(w=torch.empty(0, device="cuda"), g=torch.empty(0, device="cuda"),
+                     m=torch.empty(0, dtype=torch.uint8, device="cuda"), v=torch.empty(0, dtype=torch.uint8, device="cuda"),
+                     scale_m_in=one(), scale_v_in=one(), scale_m_out=one(), scale_v_out=one(),
+                     amax_m=torch.full((1,), 5.0, device="cuda"), amax_v=torch.full((1,), 5.0, device="cuda"))
+        B.fp8mlp_adam_step([empty], lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.0, step=1)
+        torch.cuda.synchronize()
+        assert all(float(t.abs().max()) == 0 for t in g)
+        assert empty["amax_m"].item() == 0 and empty["amax_v"].item() == 0
+        assert B.fp8mlp_status(ctx) == B.OK and B.fp8mlp_status(hb) == B.OK
+    finally:
+        B.fp8mlp_destroy(ctx)
+        B.fp8mlp_destroy(hb)
