@@ -81,7 +81,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -102,7 +102,10 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        rows = [r for t, r in self.rows if t0 <= t <= t1 and len(r) >= 8] or [r for _, r in self.rows if len(r) >= 8]
+        good = [(t, r) for t, r in self.rows if len(r) >= 8]
+        rows = [r for t, r in good if t0 <= t <= t1]
+        if not rows and good:            # a timed region shorter than the sampling period: the sample nearest to it
+            rows = [min(good, key=lambda tr: min(abs(tr[0] - t0), abs(tr[0] - t1)))[1]]
         if not rows:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
         num = lambda s: float(s) if s.replace(".", "", 1).isdigit() else None
@@ -113,7 +116,8 @@ class ClockSampler:
                 if r[col].lower().startswith("active"):
                     reasons.add(name)
         power = [v for v in (num(r[2]) for r in rows) if v is not None]
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": num(rows[0][1]),
+        masks = sorted({r[3] for r in rows})
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": num(rows[0][1]), "active_masks": masks,
                 "power_w_max": max(power) if power else None, "samples": len(rows), "reasons": sorted(reasons)}
 
 
