@@ -14,12 +14,14 @@ namespace {
 // warp streams the saved G and U (a 128-row x 64-channel bf16 box each) to the epilogue.
 constexpr int kGuSlots = 2;
 constexpr int kGuSlotBytes = 2 * kBoxBytes;
-template <bool PAIR, int EPI> struct Plan;
-template <int EPI> struct Plan<false, EPI> {
+// WIDEN (CTA pairs, plain epilogues): a 256 x 512 tile - both accumulators belong to one tile, the A block
+// of a stage is loaded once for two B blocks (a quarter less operand traffic), the epilogue is not overlapped.
+template <bool PAIR, int EPI, bool WIDEN> struct Plan;
+template <int EPI, bool WIDEN> struct Plan<false, EPI, WIDEN> {
     static constexpr int kStages = EPI == EPI_SWIGLU_BWD ? 3 : 4, kStageBytes = 3 * kBoxBytes, kTileM = 128;
 };
-template <int EPI> struct Plan<true, EPI> {
-    static constexpr int kStages = EPI == EPI_SWIGLU_BWD ? 4 : 6, kStageBytes = 2 * kBoxBytes, kTileM = 256;
+template <int EPI, bool WIDEN> struct Plan<true, EPI, WIDEN> {
+    static constexpr int kStages = (EPI == EPI_SWIGLU_BWD || WIDEN) ? 4 : 6, kStageBytes = (WIDEN ? 3 : 2) * kBoxBytes, kTileM = 256;
 };
 constexpr int kMaxStages = 6;
 
@@ -35,9 +37,9 @@ struct __align__(8) SmemTail {
     float s_tile[2][kBlockN];    // per-channel scales of the current tile(s)
     unsigned int amax_tile[128]; // per-channel maxima of the current tile (forward)
 };
-template <bool PAIR, int EPI>
+template <bool PAIR, int EPI, bool WIDEN>
 constexpr size_t smem_bytes() {
-    return 1024 /*alignment slack*/ + size_t(Plan<PAIR, EPI>::kStages) * Plan<PAIR, EPI>::kStageBytes +
+    return 1024 /*alignment slack*/ + size_t(Plan<PAIR, EPI, WIDEN>::kStages) * Plan<PAIR, EPI, WIDEN>::kStageBytes +
            (EPI == EPI_SWIGLU_BWD ? size_t(kGuSlots) * kGuSlotBytes : 0) + sizeof(SmemTail);
 }
 
@@ -354,14 +356,15 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
 // PAIR = false: one CTA per 128 x 256 tile.  PAIR = true: a cluster of two CTAs per 256 x 256 tile
 // (tcgen05 cta_group::2): rank r loads rows [128 r, 128 r + 128) of the A tile and of the B tile,
 // rank 0 issues the MMAs for both, and each CTA drains its own 128 rows of the accumulator.
-template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM>
+template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM, bool WIDEN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
             const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmG,
             const __grid_constant__ CUtensorMap tmU, const GemmArgs p) {
-    constexpr int kStages = Plan<PAIR, EPI>::kStages;
-    constexpr int kStageBytes = Plan<PAIR, EPI>::kStageBytes;
-    constexpr int kTileM = Plan<PAIR, EPI>::kTileM;
+    constexpr int kStages = Plan<PAIR, EPI, WIDEN>::kStages;
+    constexpr int kStageBytes = Plan<PAIR, EPI, WIDEN>::kStageBytes;
+    constexpr int kTileM = Plan<PAIR, EPI, WIDEN>::kTileM;
+    static_assert(!WIDEN || (PAIR && (EPI == EPI_F32 || EPI == EPI_BF16)), "wide tiles: CTA pairs, plain epilogues");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;         // swizzle atoms need 1024-byte alignment
@@ -428,6 +431,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         if (rank == 0) mbar_expect_tx(smem_u32(&tail->full[stage]), 2 * kStageBytes);
                         load_operand<A_MN, ELEM, true>(dst, &tmA, bar, m0, k0);
                         load_operand<B_MN, ELEM, true>(dst + kBoxBytes, tmB, bar, nb0, k0);
+                        if constexpr (WIDEN) load_operand<B_MN, ELEM, true>(dst + 2 * kBoxBytes, tmB, bar, nb0 + kBlockN, k0);
                     } else {
                         const uint32_t bar = smem_u32(&tail->full[stage]);
                         mbar_expect_tx(bar, kStageBytes);
@@ -446,7 +450,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             bool ok = true;
             int it = 0;
             for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step, ++it) {
-                const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
+                const uint32_t acc = WIDEN ? 0u : (it & 1), acc_phase = WIDEN ? (it & 1) : ((it >> 1) & 1);
                 if (!mbar_wait(smem_u32(&tail->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, p.status)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kBlockN;
@@ -460,7 +464,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         const uint64_t da = smem_desc<A_MN, ELEM>(a_addr + k * k_step_bytes<A_MN, ELEM>());
                         const uint64_t db = smem_desc<B_MN, ELEM>(b_addr + k * k_step_bytes<B_MN, ELEM>());
                         const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
-                        if constexpr (ELEM == 1) {
+                        if constexpr (WIDEN) {       // second half of the 512 columns: same A, the stage's other B block
+                            const uint64_t db1 = smem_desc<B_MN, ELEM>(b_addr + kBoxBytes + k * k_step_bytes<B_MN, ELEM>());
+                            umma_f8_pair(d_tmem, da, db, p.idesc, accum);
+                            umma_f8_pair(d_tmem + kBlockN, da, db1, p.idesc, accum);
+                        } else if constexpr (ELEM == 1) {
                             if constexpr (PAIR) umma_f8_pair(d_tmem, da, db, p.idesc, accum); else umma_f8(d_tmem, da, db, p.idesc, accum);
                         } else {
                             if constexpr (PAIR) umma_f16_pair(d_tmem, da, db, p.idesc, accum); else umma_f16(d_tmem, da, db, p.idesc, accum);
@@ -519,7 +527,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             tile_coords(p, tile, m_tile, n_tile);
             const int m = m_tile * kTileM + static_cast<int>(rank) * kBlockM + row;
             const int n0 = n_tile * p.n_tile_cols;
-            const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
+            const uint32_t acc = WIDEN ? 0u : (it & 1), acc_phase = WIDEN ? (it & 1) : ((it >> 1) & 1);
             if constexpr (EPI == EPI_SWIGLU_FWD) {
                 if (et < 128) {
                     tail->s_tile[0][et] = (n0 + et) < p.N ? p.s_h[n0 + et] : 1.0f;
@@ -536,8 +544,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 if (p.row_s != nullptr)
                     dq = __fmul_rn(inv_or_one(p.s0), m < p.M ? __fdiv_rn(1.0f, p.row_s[m]) : 1.0f);
                 epilogue_f32(p, taddr, half, m, n0, dq);
+                if constexpr (WIDEN) epilogue_f32(p, taddr + kBlockN, half, m, n0 + kBlockN, dq);
             } else if constexpr (EPI == EPI_BF16) {
                 epilogue_bf16(p, taddr, half, m, n0, dq0);
+                if constexpr (WIDEN) epilogue_bf16(p, taddr + kBlockN, half, m, n0 + kBlockN, dq0);
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
                 epilogue_swiglu_fwd(p, tail, taddr, lane, half, m, n0, dq0);
             } else {
@@ -603,10 +613,10 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM>
+template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM, bool WIDEN = false>
 int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorMap& tmB1, const GemmArgs& args,
                 int64_t tiles, int sm_count, cudaStream_t st) {
-    constexpr size_t kSmem = smem_bytes<PAIR, EPI>();
+    constexpr size_t kSmem = smem_bytes<PAIR, EPI, WIDEN>();
     // the saved activations [M, 2f] bf16 as two matrices of f columns: G, and U starting f elements in
     CUtensorMap tmG = tmA, tmU = tmA;
     if (EPI == EPI_SWIGLU_BWD) {
@@ -632,12 +642,12 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
         cfg.numAttrs = 1;
     }
     std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(kSmem));
         if (PAIR && attr_err == cudaSuccess) {
             // how many CTA pairs the device can hold at once (one CTA per SM, pairs on neighbouring SMs)
             cfg.gridDim = dim3(static_cast<unsigned>(sm_count) & ~1u);
-            attr_err = cudaOccupancyMaxActiveClusters(&max_clusters, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM>, &cfg);
+            attr_err = cudaOccupancyMaxActiveClusters(&max_clusters, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN>, &cfg);
         }
     });
     FP8MLP_CUDA_CHECK(attr_err);
@@ -649,14 +659,14 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
         grid = tiles < sm_count ? tiles : sm_count;
     }
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
-    FP8MLP_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM>, tmA, tmB0, tmB1, tmG, tmU, args));
+    FP8MLP_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN>, tmA, tmB0, tmB1, tmG, tmU, args));
     count_launch();
     return FP8MLP_OK;
 }
 
 }  // namespace
 
-size_t gemm_smem_bytes() { return smem_bytes<true, EPI_F32>(); }
+size_t gemm_smem_bytes() { return smem_bytes<true, EPI_F32, false>(); }
 
 int make_tmap(CUtensorMap* map, const void* base, int elem_bytes, bool mn_major, uint64_t inner, uint64_t outer,
               uint64_t row_stride_bytes) {
@@ -688,6 +698,12 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     const bool pair = args.pair_mode == 1 || (args.pair_mode == 0 && args.M > kBlockM);
     const int tile_m = pair ? 2 * kBlockM : kBlockM;
     args.num_m_tiles = (args.M + tile_m - 1) / tile_m;
+    // 256 x 512 tiles for the bf16-output GEMMs on CTA pairs with at least 512 output columns (GEMM-2, dgrad-1).  The
+    // fp32-output weight gradients keep 256 x 256 tiles: their epilogue (four times the bytes) would sit in the open
+    // and their tile counts divide worse over the CTA pairs; measured slower with wide tiles.
+    const bool widen = pair && args.elem_bytes != 2 && ((epi == EPI_BF16 && args.wide_tiles != 2) || (epi == EPI_F32 && args.wide_tiles == 1)) &&
+                       args.n_tile_cols == kBlockN && args.N >= 2 * kBlockN;
+    if (widen) args.n_tile_cols = 2 * kBlockN;
     args.num_n_tiles = (args.N + args.n_tile_cols - 1) / args.n_tile_cols;
     const int elem = args.elem_bytes == 2 ? 2 : 1;
     const int kblk = kBlockK / elem;     // contraction elements per stage
@@ -709,6 +725,16 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     const int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
     if (tiles == 0 || args.num_k_blocks == 0) return FP8MLP_OK;
 
+#define FP8MLP_DISPATCH_WIDE(E, AM, BM)                                                                     \
+    if (widen && epi == E && a_mn == AM && b_mn == BM)                                                      \
+        return launch_inst<E, AM, BM, true, 1, true>(tmA, tmB0, tmB1, args, tiles, sm_count, st);
+    FP8MLP_DISPATCH_WIDE(EPI_F32, false, false)
+    FP8MLP_DISPATCH_WIDE(EPI_F32, false, true)
+    FP8MLP_DISPATCH_WIDE(EPI_F32, true, false)
+    FP8MLP_DISPATCH_WIDE(EPI_F32, true, true)
+    FP8MLP_DISPATCH_WIDE(EPI_BF16, false, false)
+    FP8MLP_DISPATCH_WIDE(EPI_BF16, false, true)
+#undef FP8MLP_DISPATCH_WIDE
 #define FP8MLP_DISPATCH(E, AM, BM, EL)                                                                     \
     if (epi == E && a_mn == AM && b_mn == BM && elem == EL)                                                \
         return pair ? launch_inst<E, AM, BM, true, EL>(tmA, tmB0, tmB1, args, tiles, sm_count, st)         \

@@ -45,6 +45,7 @@ struct GemmArgs {
     int group_m;            // m-tiles per rasterisation band
     int pair_mode;          // 0: CTA pairs when M > 128; 1: always CTA pairs; 2: always single CTAs
     int elem_bytes;         // operand element size: 1 (FP8, default) or 2 (bf16; a_fmt = b_fmt = 1)
+    int wide_tiles;         // 256 x 512 tiles: 0 = for bf16 outputs (default), 1 = for fp32 outputs too, 2 = never
     uint32_t idesc;
     int* status;
 
