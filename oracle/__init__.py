@@ -20,7 +20,7 @@ _ADAM_SRC = _HERE / "fp8adam_oracle.c"
 _ADAM_LIB = _HERE / "liboracle_adam.so"
 
 E4M3, E5M2 = 0, 1
-FLAG_SMOOTH, FLAG_Q_IDENTITY, FLAG_NO_BF16, FLAG_H_BF16 = 1, 2, 4, 8
+FLAG_SMOOTH, FLAG_Q_IDENTITY, FLAG_NO_BF16, FLAG_H_BF16, FLAG_GU_FP8 = 1, 2, 4, 8, 16
 SCALE_GIVEN, SCALE_CURRENT = 0, 1
 
 _lib = None
@@ -172,11 +172,11 @@ def swiglu_grad(u: float, g: float, dh: float):
 
 
 def forward(x_bf16, W1, W2, W3, *, flags: int = FLAG_SMOOTH, scale_mode: int = SCALE_CURRENT,
-            sx=None, sw12=None, s_h=None, sw3=None, want_float_operands: bool = False) -> dict:
+            sx=None, sw12=None, s_h=None, sw3=None, sgu=None, want_float_operands: bool = False) -> dict:
     """Forward of the block.  x_bf16: uint16 [T,d]; W1,W2 [d,f]; W3 [f,d] float32.
 
-    In SCALE_GIVEN mode sx, sw12, s_h[f], sw3 must be supplied.  Returns every
-    intermediate the CUDA path can be compared on.
+    In SCALE_GIVEN mode sx, sw12, s_h[f], sw3 (and sgu with FLAG_GU_FP8) must be supplied.  Returns
+    every intermediate the CUDA path can be compared on.
     """
     x_bf16 = np.ascontiguousarray(x_bf16, dtype=np.uint16)
     W1, W2, W3 = _f32(W1), _f32(W2), _f32(W3)
@@ -188,6 +188,11 @@ def forward(x_bf16, W1, W2, W3, *, flags: int = FLAG_SMOOTH, scale_mode: int = S
     if scale_mode == SCALE_GIVEN:
         assert None not in (sx, sw12, sw3) and s_h is not None and sh.shape == (f,)
     am = [C.c_float(0) for _ in range(4)]
+    gu_fp8 = bool(flags & FLAG_GU_FP8)
+    if gu_fp8 and scale_mode == SCALE_GIVEN:
+        assert sgu is not None
+    c_sgu, a_gu = C.c_float(sgu or 0), C.c_float(0)
+    GUq = np.empty((T, 2 * f), np.uint8) if gu_fp8 else None
     r = dict(
         amax_h=np.empty(f, np.float32), Xq=np.empty((T, d), np.uint8), W12q=np.empty((d, 2 * f), np.uint8),
         W3q=np.empty((f, d), np.uint8), Hq=np.empty((T, f), np.uint8), G=np.empty((T, f), np.uint16),
@@ -206,9 +211,12 @@ def forward(x_bf16, W1, W2, W3, *, flags: int = FLAG_SMOOTH, scale_mode: int = S
         _p(r["Xq"]), _p(r["W12q"]), _p(r["W3q"]), _p(r["Hq"]), _p(r["G"]), _p(r["U"]), _p(r["H"]),
         _p(r["Y_bits"]), _p(r["Y"]),
         _p(fl.get("xq_f")), _p(fl.get("w12q_f")), _p(fl.get("w3q_f")), _p(fl.get("hq_f")),
-        _p(fl.get("G_f32")), _p(fl.get("U_f32")))
+        _p(fl.get("G_f32")), _p(fl.get("U_f32")),
+        C.byref(c_sgu), C.byref(a_gu), _p(GUq))
     assert rc == 0
     r.update(fl)
+    if gu_fp8:
+        r.update(GUq=GUq, sgu=float(c_sgu.value), amax_gu=float(a_gu.value))
     r.update(sx=float(c_sx.value), sw12=float(c_sw12.value), sw3=float(c_sw3.value), s_h=sh,
              amax_x=float(am[0].value), amax_w1=float(am[1].value), amax_w2=float(am[2].value),
              amax_w3=float(am[3].value), flags=flags, T=T, d=d, f=f)
@@ -234,7 +242,8 @@ def backward(fwd: dict, dy_bf16, *, scale_mode: int = SCALE_CURRENT, sdy=None, s
         _p(fwd["G"]), _p(fwd["U"]), _p(fwd.get("G_f32")), _p(fwd.get("U_f32")),
         C.c_float(fwd["sx"]), C.c_float(fwd["sw12"]), _p(fwd["s_h"]), C.c_float(fwd["sw3"]),
         C.byref(c_sdy), C.byref(c_sdz), C.byref(a_dy), C.byref(a_dz),
-        _p(r["dYq"]), _p(r["dZq"]), _p(r["dX_bits"]), _p(r["dX"]), _p(r["dW1"]), _p(r["dW2"]), _p(r["dW3"]))
+        _p(r["dYq"]), _p(r["dZq"]), _p(r["dX_bits"]), _p(r["dX"]), _p(r["dW1"]), _p(r["dW2"]), _p(r["dW3"]),
+        _p(fwd.get("GUq")), C.c_float(fwd.get("sgu", 1.0)))
     assert rc == 0
     r.update(sdy=float(c_sdy.value), sdz=float(c_sdz.value), amax_dy=float(a_dy.value), amax_dz=float(a_dz.value))
     return r

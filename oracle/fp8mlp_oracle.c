@@ -51,6 +51,9 @@
 #define ORC_FLAG_H_BF16      8u  /* the paper's "SwiGLU output in BF16" variant (Section 4.3): the
                                     last linear layer is not quantised - its input H, its weight W3
                                     and the dY it meets in backward are bf16; everything else FP8   */
+#define ORC_FLAG_GU_FP8     16u  /* the activations kept for backward, G and U, are stored as E4M3
+                                    codes with one per-tensor scale instead of bf16 (the paper does
+                                    not say how they are kept: a reading, offered as an option)     */
 
 #define ORC_SCALE_GIVEN   0
 #define ORC_SCALE_CURRENT 1
@@ -286,7 +289,9 @@ void orc_swiglu_grad(float u_lin, float g_gate, float dh, float* du, float* dg) 
  *          [0,f), linear W1 in [f,2f)), W3q [f,d], Hq [T,f]; saved G,U (bf16 bits, [T,f]);
  *          H fp32 (unscaled SwiGLU output); Y (bf16 bits) and Y as fp32.
  * READING: W1 and W2 share one scale (they are one concatenated operand).
- * READING: saved activations for backward are the bf16-rounded G and U.
+ * READING: saved activations for backward are the bf16-rounded G and U; with ORC_FLAG_GU_FP8 they
+ *          are GUq [T,2f] = Q_e4m3(sgu * [G | U]) instead, sgu one scale for both (448 / max(|G|,|U|)
+ *          in current-amax mode), and backward takes G~ = decode(code) * (1 / sgu).
  * READING: with Smooth off, H gets one per-tensor scale sh = 448/max_i amax_h[i] held in
  *          every s_h[i]; W3 is quantised unscaled and 1/sh joins the output dequantisation.
  */
@@ -297,7 +302,8 @@ int orc_forward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode,
                 uint8_t* Xq, uint8_t* W12q, uint8_t* W3q, uint8_t* Hq,
                 uint16_t* G_bf16, uint16_t* U_bf16, float* H_f32,
                 uint16_t* Y_bf16, float* Y_f32,
-                float* xq_f, float* w12q_f, float* w3q_f, float* hq_f, float* G_f32, float* U_f32) {
+                float* xq_f, float* w12q_f, float* w3q_f, float* hq_f, float* G_f32, float* U_f32,
+                float* sgu, float* amax_gu, uint8_t* GUq) {
     const int smooth = (flags & ORC_FLAG_SMOOTH) != 0;
     float* xf   = (float*)malloc(sizeof(float) * T * d);
     float* xq   = (float*)malloc(sizeof(float) * T * d);
@@ -334,6 +340,22 @@ int orc_forward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode,
     const float inv_sx = 1.0f / *sx, inv_sw12 = 1.0f / *sw12;
     const float dq1 = inv_sx * inv_sw12;
     for (int64_t i = 0; i < f; ++i) ah[i] = 0.0f;
+    if (flags & ORC_FLAG_GU_FP8) {
+        /* G and U kept as E4M3 codes: their common maximum, the scale, the codes */
+        float agu = 0.0f;
+        for (int64_t j = 0; j < T * f; ++j) {
+            float a = fabsf(accG[j] * dq1); if (a > agu) agu = a;
+            a = fabsf(accU[j] * dq1);       if (a > agu) agu = a;
+        }
+        if (amax_gu) *amax_gu = agu;
+        if (scale_mode == ORC_SCALE_CURRENT) *sgu = orc_scale_from_amax(ORC_E4M3, agu);
+        if (GUq)
+            for (int64_t t = 0; t < T; ++t)
+                for (int64_t i = 0; i < f; ++i) {
+                    quant1(ORC_E4M3, accG[t * f + i] * dq1, *sgu, flags, &GUq[t * 2 * f + i]);
+                    quant1(ORC_E4M3, accU[t * f + i] * dq1, *sgu, flags, &GUq[t * 2 * f + f + i]);
+                }
+    }
     for (int64_t t = 0; t < T; ++t)
         for (int64_t i = 0; i < f; ++i) {
             float g = accG[t * f + i] * dq1;
@@ -430,7 +452,8 @@ int orc_forward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode,
 
 /* ------------------------------------------------------------------ backward
  * Takes what forward left behind: codes Xq, W12q, W3q, Hq, saved G,U (bf16 bits, or fp32
- * arrays G_f32/U_f32 when ORC_FLAG_NO_BF16), and the forward scales.
+ * arrays G_f32/U_f32 when ORC_FLAG_NO_BF16, or E4M3 codes GUq with their scale when
+ * ORC_FLAG_GU_FP8), and the forward scales.
  * READING: every Q is straight-through and s_i is a constant; weights and activations
  * keep their E4M3 codes in the backward GEMMs, only dY and dZ = [dG|dU] are E5M2.
  * The header above lists what pins this.
@@ -447,7 +470,8 @@ int orc_backward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode
                  float sx, float sw12, const float* s_h, float sw3,
                  float* sdy, float* sdz, float* amax_dy, float* amax_dz,
                  uint8_t* dYq, uint8_t* dZq /*[T,2f]: dG | dU*/,
-                 uint16_t* dX_bf16, float* dX_f32, float* dW1, float* dW2, float* dW3) {
+                 uint16_t* dX_bf16, float* dX_f32, float* dW1, float* dW2, float* dW3,
+                 const uint8_t* GUq, float sgu) {
     const int smooth = (flags & ORC_FLAG_SMOOTH) != 0;
     const int qid = (flags & ORC_FLAG_Q_IDENTITY) != 0;
     float* dyf  = (float*)malloc(sizeof(float) * T * d);
@@ -506,8 +530,15 @@ int orc_backward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode
         for (int64_t i = 0; i < f; ++i) {
             float dht = accH[t * f + i] * dqh;
             float dh = smooth ? dht * s_h[i] : dht;
-            float g = (flags & ORC_FLAG_NO_BF16) ? G_f32[t * f + i] : orc_bf16_to_f32(G_bf16[t * f + i]);
-            float u = (flags & ORC_FLAG_NO_BF16) ? U_f32[t * f + i] : orc_bf16_to_f32(U_bf16[t * f + i]);
+            float g, u;
+            if (flags & ORC_FLAG_GU_FP8) {          /* kept as E4M3 codes with the scale sgu */
+                g = orc_decode(ORC_E4M3, GUq[t * 2 * f + i]) * (1.0f / sgu);
+                u = orc_decode(ORC_E4M3, GUq[t * 2 * f + f + i]) * (1.0f / sgu);
+            } else if (flags & ORC_FLAG_NO_BF16) {
+                g = G_f32[t * f + i]; u = U_f32[t * f + i];
+            } else {
+                g = orc_bf16_to_f32(G_bf16[t * f + i]); u = orc_bf16_to_f32(U_bf16[t * f + i]);
+            }
             float du, dg;
             orc_swiglu_grad(u, g, dh, &du, &dg);
             dG[t * f + i] = dg;

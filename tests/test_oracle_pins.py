@@ -422,3 +422,78 @@ def test_h_bf16_variant_last_layer_runs_in_bf16():
     cos = lambda a, b: float((a * b).sum() / np.sqrt((a * a).sum() * (b * b).sum()))
     for got, ref in ((bw["dX"], dX64), (bw["dW1"], dW1_64), (bw["dW2"], dW2_64), (bw["dW3"], dW3_64)):
         assert cos(got.astype(np.float64), ref) > 0.99
+
+
+def test_gu_fp8_option_saved_activations_as_e4m3_codes():
+    """Option (the paper does not say how the SwiGLU inputs are kept for backward): G and U are stored as
+    E4M3 codes with one per-tensor scale.  Pins: the maximum is numpy's over the fp32 G, U; the scale is
+    448 / max; the codes are a library's E4M3 cast of sgu * [G | U]; the decoded values lie within half a
+    spacing of G, U; the forward result does not change; backward's dZ codes equal a brute-force fp64
+    evaluation of the SwiGLU derivative on the decoded activations; and the gradients still point where
+    the fp64 block's do."""
+    w = wl.make("gu8", 11, 40, 64, 144, w_std=0.08)
+    fl = FLAG_SMOOTH | oracle.FLAG_GU_FP8
+    ref = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=FLAG_SMOOTH, want_float_operands=True)
+    fw = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=fl, want_float_operands=True)
+    G, U = fw["G_f32"], fw["U_f32"]
+    agu = max(np.abs(G).max(), np.abs(U).max())
+    assert fw["amax_gu"] == np.float32(agu)
+    assert fw["sgu"] == np.float32(448.0) / np.float32(agu)
+    scaled = np.concatenate([G, U], axis=1) * np.float32(fw["sgu"])
+    lib_codes = torch.from_numpy(scaled).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(fw["GUq"], lib_codes)
+    dec = _torch_decode(E4M3, fw["GUq"]).astype(np.float64) / np.float64(fw["sgu"])
+    true = np.concatenate([G, U], axis=1).astype(np.float64)
+    # 3 mantissa bits: half a spacing is 2^-4 relative in the normal range, 2^-10 / sgu absolute below it
+    assert np.all(np.abs(dec - true) <= np.abs(true) * 2.0 ** -4 + 2.0 ** -10 / fw["sgu"] + 1e-12)
+    for k in ("Xq", "W12q", "W3q", "Hq", "Y_bits"):
+        assert np.array_equal(fw[k], ref[k])
+    # backward: the derivative is taken at the decoded activations
+    bw = oracle.backward(fw, w.dY)
+    inv = np.float32(1.0) / np.float32(fw["sgu"])
+    g = (_torch_decode(E4M3, fw["GUq"][:, :144]) * inv).astype(np.float64)
+    u = (_torch_decode(E4M3, fw["GUq"][:, 144:]) * inv).astype(np.float64)
+    dyq = _torch_decode(E5M2, bw["dYq"]).astype(np.float64) / bw["sdy"]
+    w3q = _torch_decode(E4M3, fw["W3q"]).astype(np.float64) / fw["sw3"]
+    dh = (dyq @ w3q.T) * fw["s_h"].astype(np.float64)[None, :]
+    sig = 1.0 / (1.0 + np.exp(-g))
+    dz = np.concatenate([dh * u * sig * (1.0 + g * (1.0 - sig)), dh * g * sig], axis=1)
+    assert abs(bw["amax_dz"] - np.abs(dz).max()) <= 1e-5 * np.abs(dz).max()
+    got = _torch_decode(E5M2, bw["dZq"]).astype(np.float64) / bw["sdz"]
+    # E5M2 spacing is 2^-2 relative: the code of the fp64 value or, on a rounding tie-break, its neighbour
+    assert np.all(np.abs(got - dz) <= np.abs(dz) * 2.0 ** -3 * 1.001 + 2.0 ** -17 / bw["sdz"])
+    want = torch.from_numpy((dz * bw["sdz"]).astype(np.float32)).to(torch.float8_e5m2).view(torch.uint8).numpy()
+    assert np.mean(want != bw["dZq"]) < 2e-3
+    # against the bf16-saved run and the unquantised block
+    bw_ref = oracle.backward(ref, w.dY)
+    x = wl.bf16_bits_to_f32(w.x).astype(np.float64)
+    dy = wl.bf16_bits_to_f32(w.dY).astype(np.float64)
+    dX64, dW1_64, dW2_64, dW3_64 = oracle.mlp_f64_backward(x, w.W1, w.W2, w.W3, dy)
+    assert np.array_equal(bw["dW3"], bw_ref["dW3"])              # does not involve G, U
+    cos = lambda a, b: float((a * b).sum() / np.sqrt((a * a).sum() * (b * b).sum()))
+    for got_, r64 in ((bw["dX"], dX64), (bw["dW1"], dW1_64), (bw["dW2"], dW2_64)):
+        assert cos(got_.astype(np.float64), r64) > 0.99
+
+
+def test_gu_fp8_option_is_exact_when_the_activations_are_representable():
+    """When every G and U is a small integer (exact in E4M3 at a power-of-two scale and in bf16), keeping
+    them as E4M3 codes or as bf16 gives bit-identical gradients; a wrong direction of the scale, a swapped
+    G / U half or a dropped dequantisation would not."""
+    T, d, f = 8, 16, 32
+    rng = np.random.default_rng(5)
+    x = np.zeros((T, d), np.float32)
+    x[np.arange(T), rng.integers(0, d, T)] = 1.0                    # one-hot tokens: G, U are rows of W2, W1
+    W1 = rng.integers(-7, 8, (d, f)).astype(np.float32)
+    W2 = rng.integers(-7, 8, (d, f)).astype(np.float32)
+    W3 = rng.standard_normal((f, d)).astype(np.float32) * 0.1
+    dY = wl.f32_to_bf16_bits(rng.standard_normal((T, d)).astype(np.float32))
+    xb = wl.f32_to_bf16_bits(x)
+    given = dict(scale_mode=SCALE_GIVEN, sx=1.0, sw12=16.0, s_h=np.ones(f, np.float32), sw3=64.0)
+    a = oracle.forward(xb, W1, W2, W3, flags=0, **given)
+    b = oracle.forward(xb, W1, W2, W3, flags=oracle.FLAG_GU_FP8, sgu=4.0, **given)
+    assert np.array_equal(_torch_decode(E4M3, b["GUq"][:, :f]) / 4.0, wl.bf16_bits_to_f32(a["G"]))
+    assert np.array_equal(_torch_decode(E4M3, b["GUq"][:, f:]) / 4.0, wl.bf16_bits_to_f32(a["U"]))
+    ba = oracle.backward(a, dY, scale_mode=SCALE_GIVEN, sdy=64.0, sdz=8.0)
+    bb = oracle.backward(b, dY, scale_mode=SCALE_GIVEN, sdy=64.0, sdz=8.0)
+    for k in ("dZq", "dX_bits", "dW1", "dW2", "dW3"):
+        assert np.array_equal(ba[k], bb[k]), k
