@@ -353,8 +353,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                   "what": "quantise x + gate/up GEMM with SwiGLU epilogue + down GEMM on merged FP8 weights"}
     B.fp8mlp_destroy(ctx)
     # the same step with plain per-tensor FP8 for the SwiGLU output (Smooth-SwiGLU off), for the cost of smoothing
-    plain, hbf16 = None, None
-    for variant_flags in ((B.SAVE_FOR_BWD, B.H_BF16 | B.SAVE_FOR_BWD) if rank == 0 else ()):
+    plain, hbf16, gu8 = None, None, None
+    for variant_flags in ((B.SAVE_FOR_BWD, B.H_BF16 | B.SAVE_FOR_BWD, B.SMOOTH | B.SAVE_FOR_BWD | B.GU_FP8) if rank == 0 else ()):
         ctx0 = B.fp8mlp_create(T, d, f, variant_flags)
         sc0, am0 = B.new_scales(f), B.new_amax(f)
 
@@ -377,6 +377,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         res = {"ms_per_step": round(v_ms, 4), "tflops": round(job_tflops(T, d, f, 1, v_ms), 1)}
         if variant_flags & B.H_BF16:
             hbf16 = res
+        elif variant_flags & B.GU_FP8:
+            res["saved_activation_bytes"] = 2 * T * f
+            gu8 = res
         else:
             plain = res
         B.fp8mlp_destroy(ctx0)
@@ -441,9 +444,11 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                                   "step_with_just_in_time_scales": jit,
                                   "step_with_smooth_swiglu_off": plain,
                                   "step_with_swiglu_output_in_bf16": hbf16,
+                                  "step_with_saved_activations_in_fp8": gu8,
                                   "note": "Adam with E4M3/E5M2 moments on W1, W2, W3, and the inference form of "
                                           "Smooth-SwiGLU; the same step with plain per-tensor FP8 and with the last layer in "
-                                          "bf16 (the other rows of the paper's throughput table); none is included in value"}
+                                          "bf16 (the other rows of the paper's throughput table); the Smooth-SwiGLU step with G, U kept for "
+                                          "backward as E4M3 codes instead of bf16; none is included in value"}
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(out))

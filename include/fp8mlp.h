@@ -54,9 +54,13 @@ enum { FP8MLP_BF16 = 0, FP8MLP_F32 = 1 };
 enum {
     FP8MLP_SMOOTH = 1,       /* per-channel Smooth-SwiGLU scales; without it one per-tensor scale for H */
     FP8MLP_SAVE_FOR_BWD = 2, /* forward keeps bf16 G = x W2 and U = x W1 for backward               */
-    FP8MLP_H_BF16 = 4        /* the paper's "SwiGLU output in BF16" variant (Section 4.3): the last linear
+    FP8MLP_H_BF16 = 4,       /* the paper's "SwiGLU output in BF16" variant (Section 4.3): the last linear
                                 layer is not quantised - H, W3 and, in backward, dY are bf16 operands and
                                 scales.h / scales.w3 / scales.dy are unused; not with FP8MLP_SMOOTH        */
+    FP8MLP_GU_FP8 = 8        /* with FP8MLP_SAVE_FOR_BWD: G and U are kept as E4M3 codes Q(sgu [G | U]) with one
+                                per-tensor scale (scales.gu, amax.gu) instead of bf16 - half the saved bytes.
+                                The paper does not say how these activations are kept; this is an option in
+                                the spirit of its FP8 memory savings (Section 5).  Not with FP8MLP_H_BF16     */
 };
 enum {
     FP8MLP_SCALE_GIVEN = 0,              /* delayed scaling: use the scale buffers as they are  */
@@ -67,7 +71,7 @@ enum { /* fp8mlp_workspace: internal buffers, for inspection by tests */
     FP8MLP_WS_W12Q = 1, /* E4M3 [d,2f]  quantised [W2 | W1]: gate columns [0,f), linear [f,2f) */
     FP8MLP_WS_W3Q = 2,  /* E4M3 [f,d]   quantised diag(s^-1) W3                        */
     FP8MLP_WS_HQ = 3,   /* E4M3 [T,f]   Q(s_i * SwiGLU)                                */
-    FP8MLP_WS_GU = 4,   /* bf16 [T,2f]  saved G | U                                    */
+    FP8MLP_WS_GU = 4,   /* bf16 [T,2f]  saved G | U  (E4M3 [T,2f] with FP8MLP_GU_FP8)  */
     FP8MLP_WS_DYQ = 5,  /* E5M2 [T,d]   quantised dY                                   */
     FP8MLP_WS_DZQ = 6,  /* E5M2 [T,2f]  quantised [dG | dU]                            */
     FP8MLP_WS_HB = 7,   /* bf16 [T,f]   SwiGLU output, FP8MLP_H_BF16 contexts only      */
@@ -96,9 +100,11 @@ enum { /* phases of one step, for fp8mlp_profile_read (SMOOTH-mode kernel sequen
  *   amax.h[f]  : per-channel max |SwiGLU output| before scaling (Section 4.4, steps 1-2).
  *   amax.w3    : max |W3[i,j] / s_i|  (the tensor that is actually quantised).
  *   w12 / dz   : one scale for the concatenated [W2|W1] and [dG|dU] operands; amax of W1 and
- *                W2 are still reported separately. */
-typedef struct { float *x, *w12, *w3, *dy, *dz, *h; } fp8mlp_scales;
-typedef struct { float *x, *w1, *w2, *w3, *dy, *dz, *h; } fp8mlp_amax;
+ *                W2 are still reported separately.
+ *   gu         : FP8MLP_GU_FP8 contexts only (may be NULL otherwise): scale of the saved [G | U] and
+ *                max(|G|, |U|). */
+typedef struct { float *x, *w12, *w3, *dy, *dz, *h, *gu; } fp8mlp_scales;
+typedef struct { float *x, *w1, *w2, *w3, *dy, *dz, *h, *gu; } fp8mlp_amax;
 
 /* Creates a context for T <= T_max tokens.  Allocates its workspace on the current device
  * (about T_max*(2d + 7f) + 3*d*f bytes).  Host call; may synchronise. */
@@ -148,6 +154,7 @@ FP8MLP_API int fp8mlp_quantize(const void* src, int src_dtype, int64_t rows, int
  *   x, w3, dy : scale = fmt_max / amax.     w12 : 448 / max(amax.w1, amax.w2).
  *   h[i]      : Smooth on: largest power of two p with p * amax.h[i] <= 448; off: 448 / max_i amax.h[i].
  *   dz        : largest power of two p with p * amax.dz <= 57344.
+ *   gu        : 448 / amax.gu.
  * A zero or non-finite amax gives scale 1.  Members of `amax` that are NULL are skipped together
  * with their scale. */
 FP8MLP_API int fp8mlp_update_scales(fp8mlp_ctx* ctx, const fp8mlp_amax* amax, fp8mlp_scales* scales, void* stream);
@@ -160,7 +167,9 @@ FP8MLP_API int fp8mlp_update_scales(fp8mlp_ctx* ctx, const fp8mlp_amax* amax, fp
  *   SCALE_GIVEN: `scales` are read; `amax` (nullable, members nullable) receives this call's maxima.
  *   SCALE_FROM_CURRENT_AMAX: both structs must be complete; scales.x/w12/h/w3 are overwritten from
  *   this call's data first (runs step 1-2 twice: once for the per-channel maxima, once for the codes).
- *   With FP8MLP_SAVE_FOR_BWD in the context flags, bf16 G and U are kept for fp8mlp_backward. */
+ *   With FP8MLP_SAVE_FOR_BWD in the context flags, bf16 G and U are kept for fp8mlp_backward; with
+ *   FP8MLP_GU_FP8 as well they are kept as Q_e4m3([G | U] sgu) (scales.gu required; amax.gu = max(|G|, |U|),
+ *   required in SCALE_FROM_CURRENT_AMAX mode, which derives sgu = 448 / amax.gu first). */
 FP8MLP_API int fp8mlp_forward(fp8mlp_ctx* ctx, int64_t T, const void* x_bf16,
                    const float* W1, const float* W2, const float* W3,
                    int scale_mode, fp8mlp_scales* scales, fp8mlp_amax* amax,
@@ -174,7 +183,8 @@ FP8MLP_API int fp8mlp_forward(fp8mlp_ctx* ctx, int64_t T, const void* x_bf16,
  *   dX = dZq [W2q|W1q]^T / (sdz sw12)  -> bf16 [T,d]
  *   [dW2|dW1] = Xq^T dZq / (sx sdz)    -> fp32 [d,f] each, overwritten
  *   dW3[i,:] = (Hq^T dYq)[i,:] / (sdy s_i) -> fp32 [f,d], overwritten
- * Every Q is straight-through and s is a constant.  scale_mode as in forward, for dy and dz. */
+ * Every Q is straight-through and s is a constant.  scale_mode as in forward, for dy and dz.
+ * FP8MLP_GU_FP8: G and U above are the decoded saved codes times 1 / sgu (scales.gu as in the forward). */
 FP8MLP_API int fp8mlp_backward(fp8mlp_ctx* ctx, int64_t T, const void* dy_bf16,
                     int scale_mode, fp8mlp_scales* scales, fp8mlp_amax* amax,
                     void* dx_bf16, float* dW1, float* dW2, float* dW3, void* stream);

@@ -19,7 +19,7 @@ OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_CUDA, ERR_TIMEOUT, ERR_STATE, ERR_TOO_LAR
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 E4M3, E5M2 = 0, 1
 BF16, F32 = 0, 1
-SMOOTH, SAVE_FOR_BWD, H_BF16 = 1, 2, 4
+SMOOTH, SAVE_FOR_BWD, H_BF16, GU_FP8 = 1, 2, 4, 8
 SCALE_GIVEN, SCALE_FROM_CURRENT_AMAX = 0, 1
 WS_XQ, WS_W12Q, WS_W3Q, WS_HQ, WS_GU, WS_DYQ, WS_DZQ, WS_HB, WS_W3B = range(9)
 
@@ -44,11 +44,11 @@ class Fp8MlpError(RuntimeError):
 
 
 class _Scales(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("x", "w12", "w3", "dy", "dz", "h")]
+    _fields_ = [(n, C.c_void_p) for n in ("x", "w12", "w3", "dy", "dz", "h", "gu")]
 
 
 class _Amax(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("x", "w1", "w2", "w3", "dy", "dz", "h")]
+    _fields_ = [(n, C.c_void_p) for n in ("x", "w1", "w2", "w3", "dy", "dz", "h", "gu")]
 
 
 class _AdamTensor(C.Structure):
@@ -124,13 +124,13 @@ def _check(code: int, where: str):
 
 
 def _scales(s: dict) -> _Scales:
-    return _Scales(*[(s[n].data_ptr() if s.get(n) is not None else None) for n in ("x", "w12", "w3", "dy", "dz", "h")])
+    return _Scales(*[(s[n].data_ptr() if s.get(n) is not None else None) for n in ("x", "w12", "w3", "dy", "dz", "h", "gu")])
 
 
 def _amax(a: dict | None):
     if a is None:
         return None
-    return _Amax(*[(a[n].data_ptr() if a.get(n) is not None else None) for n in ("x", "w1", "w2", "w3", "dy", "dz", "h")])
+    return _Amax(*[(a[n].data_ptr() if a.get(n) is not None else None) for n in ("x", "w1", "w2", "w3", "dy", "dz", "h", "gu")])
 
 
 def fp8mlp_launch_count() -> int:
@@ -258,13 +258,13 @@ def fp8mlp_gemm_bf16(M: int, N: int, K: int, A, a_kmajor: bool, B, b_kmajor: boo
 
 def new_scales(d_ff: int, device="cuda") -> dict:
     """Caller-owned scale buffers, initialised to 1."""
-    s = {n: torch.ones(1, dtype=torch.float32, device=device) for n in ("x", "w12", "w3", "dy", "dz")}
+    s = {n: torch.ones(1, dtype=torch.float32, device=device) for n in ("x", "w12", "w3", "dy", "dz", "gu")}
     s["h"] = torch.ones(d_ff, dtype=torch.float32, device=device)
     return s
 
 
 def new_amax(d_ff: int, device="cuda") -> dict:
-    a = {n: torch.zeros(1, dtype=torch.float32, device=device) for n in ("x", "w1", "w2", "w3", "dy", "dz")}
+    a = {n: torch.zeros(1, dtype=torch.float32, device=device) for n in ("x", "w1", "w2", "w3", "dy", "dz", "gu")}
     a["h"] = torch.zeros(d_ff, dtype=torch.float32, device=device)
     return a
 

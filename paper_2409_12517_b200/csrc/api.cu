@@ -167,7 +167,7 @@ int quantize_w12(fp8mlp_ctx* c, const float* W1, const float* W2, int mode, floa
 
 // G|U = Xq [W2q|W1q] with the SwiGLU / Smooth-SwiGLU epilogue
 int gemm1_swiglu(fp8mlp_ctx* c, int64_t T, const fp8mlp_scales* s, float* amax_h, int store, cudaStream_t st,
-                 bool save_gu = true) {
+                 bool save_gu = true, float* amax_gu = nullptr) {
     CUtensorMap tmA, tmB0, tmB1;
     FP8MLP_TRY(make_tmap_u8(&tmA, c->xq, c->d, T, c->d));
     FP8MLP_TRY(make_tmap_u8(&tmB0, c->w12q, c->f, c->d, 2 * c->f));
@@ -181,6 +181,12 @@ int gemm1_swiglu(fp8mlp_ctx* c, int64_t T, const fp8mlp_scales* s, float* amax_h
     a.hq = c->hq;
     a.hb = (c->flags & FP8MLP_H_BF16) ? c->hb : nullptr;
     a.gu = (save_gu && (c->flags & FP8MLP_SAVE_FOR_BWD)) ? c->gu : nullptr;
+    if (a.gu != nullptr && (c->flags & FP8MLP_GU_FP8)) {      // kept as E4M3 codes instead
+        a.gu8 = reinterpret_cast<uint8_t*>(c->gu);
+        a.gu = nullptr;
+        a.s_gu = s->gu;
+        a.amax_gu = reinterpret_cast<unsigned int*>(amax_gu);
+    }
     a.amax_h = reinterpret_cast<unsigned int*>(amax_h);
     return launch_gemm(EPI_SWIGLU_FWD, false, true, FP8MLP_E4M3, FP8MLP_E4M3, tmA, tmB0, tmB1, a, c->sm_count, st);
 }
@@ -210,8 +216,9 @@ int64_t fp8mlp_launch_count(void) { return g_launches.load(std::memory_order_rel
 int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_t flags) {
     if (out == nullptr) return FP8MLP_ERR_ARG;
     *out = nullptr;
-    if (flags & ~uint32_t(FP8MLP_SMOOTH | FP8MLP_SAVE_FOR_BWD | FP8MLP_H_BF16)) return FP8MLP_ERR_ARG;
+    if (flags & ~uint32_t(FP8MLP_SMOOTH | FP8MLP_SAVE_FOR_BWD | FP8MLP_H_BF16 | FP8MLP_GU_FP8)) return FP8MLP_ERR_ARG;
     if ((flags & FP8MLP_SMOOTH) && (flags & FP8MLP_H_BF16)) return FP8MLP_ERR_ARG;   // nothing to smooth: H is not quantised
+    if ((flags & FP8MLP_GU_FP8) && ((flags & FP8MLP_H_BF16) || !(flags & FP8MLP_SAVE_FOR_BWD))) return FP8MLP_ERR_ARG;
     if (T_max < 0 || d <= 0 || f <= 0 || d % 16 != 0 || f % 16 != 0) return FP8MLP_ERR_SHAPE;
     if (T_max > (1 << 30) || d > (1 << 24) || f > (1 << 24)) return FP8MLP_ERR_SHAPE;
     fp8mlp_ctx* c = new (std::nothrow) fp8mlp_ctx();
@@ -228,7 +235,7 @@ int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_
     c->bytes[FP8MLP_WS_W12Q] = d * 2 * f;
     c->bytes[FP8MLP_WS_W3Q] = f * d;
     c->bytes[FP8MLP_WS_HQ] = Tm * f;
-    c->bytes[FP8MLP_WS_GU] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * 2 * f * 2 : 16;
+    c->bytes[FP8MLP_WS_GU] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * 2 * f * ((flags & FP8MLP_GU_FP8) ? 1 : 2) : 16;
     c->bytes[FP8MLP_WS_DYQ] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * d : 16;
     c->bytes[FP8MLP_WS_DZQ] = (flags & FP8MLP_SAVE_FOR_BWD) ? Tm * 2 * f : 16;
     const bool hb16 = (flags & FP8MLP_H_BF16) != 0;
@@ -362,6 +369,7 @@ int fp8mlp_update_scales(fp8mlp_ctx* c, const fp8mlp_amax* am, fp8mlp_scales* sc
     a.amax_dy = am->dy; a.amax_dz = am->dz; a.amax_h = am->h;
     a.scale_x = sc->x; a.scale_w12 = sc->w12; a.scale_w3 = sc->w3;
     a.scale_dy = sc->dy; a.scale_dz = sc->dz; a.scale_h = sc->h;
+    if (c->flags & FP8MLP_GU_FP8) { a.amax_gu = am->gu; a.scale_gu = sc->gu; }
     a.f = c->f;
     a.smooth = (c->flags & FP8MLP_SMOOTH) ? 1 : 0;
     return run_update_scales(a, c->sm_count, static_cast<cudaStream_t>(stream));
@@ -377,6 +385,8 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
     if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX &&
         (am == nullptr || am->x == nullptr || am->w1 == nullptr || am->w2 == nullptr || am->w3 == nullptr || am->h == nullptr))
         return FP8MLP_ERR_ARG;
+    const bool gu_fp8 = (c->flags & FP8MLP_GU_FP8) != 0;
+    if (gu_fp8 && (sc->gu == nullptr || (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX && am->gu == nullptr))) return FP8MLP_ERR_ARG;
     if (!aligned16(x) || !aligned16(y) || !aligned16(W1) || !aligned16(W2) || !aligned16(W3)) return FP8MLP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool smooth = (c->flags & FP8MLP_SMOOTH) != 0;
@@ -387,12 +397,13 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
     float* a_w2 = (am && am->w2) ? am->w2 : c->dummy + 2;
     float* a_w3 = (am && am->w3) ? am->w3 : c->dummy + 3;
     float* a_h = (am && am->h) ? am->h : c->dummy + 8;
+    float* a_gu = (gu_fp8 && am && am->gu) ? am->gu : c->dummy + 7;
     c->saved_T = -1;
     c->merged = false;
 
     {
         PhaseTimer pt(c, FP8MLP_PH_MISC, st);
-        FP8MLP_TRY(zero_floats({a_x, a_w1, a_w2, a_w3}, st, a_h, f));
+        FP8MLP_TRY(zero_floats({a_x, a_w1, a_w2, a_w3, a_gu}, st, a_h, f));
     }
     {   // x -> E4M3
         PhaseTimer pt(c, FP8MLP_PH_QUANT_X, st);
@@ -443,12 +454,13 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
         // calibration pass: per-channel maxima of H, then s_i (or the per-tensor scale)
         if (T > 0) {
             PhaseTimer pt(c, FP8MLP_PH_GEMM1, st);
-            FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/0, st));
+            FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/0, st, true, a_gu));
         }
         {
             PhaseTimer pt(c, FP8MLP_PH_MISC, st);
             UpdateScalesArgs u{};
             u.amax_h = a_h; u.scale_h = sc->h; u.f = f; u.smooth = smooth ? 1 : 0;
+            if (gu_fp8) { u.amax_gu = a_gu; u.scale_gu = sc->gu; }
             FP8MLP_TRY(run_update_scales(u, c->sm_count, st));
         }
         // W3' = diag(1/s) W3 -> E4M3
@@ -459,7 +471,7 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
     if (T == 0) { c->saved_T = (c->flags & FP8MLP_SAVE_FOR_BWD) ? 0 : -1; return FP8MLP_OK; }
     {
         PhaseTimer pt(c, FP8MLP_PH_GEMM1, st);
-        FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/1, st));
+        FP8MLP_TRY(gemm1_swiglu(c, T, sc, a_h, /*store=*/1, st, true, a_gu));
     }
     // Y = Hq W3q
     PhaseTimer pt2(c, FP8MLP_PH_GEMM2, st);
@@ -565,6 +577,7 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
     if (T > 0 && (dy == nullptr || dx == nullptr)) return FP8MLP_ERR_ARG;
     if (sc->x == nullptr || sc->w12 == nullptr || sc->w3 == nullptr || sc->h == nullptr || sc->dy == nullptr || sc->dz == nullptr)
         return FP8MLP_ERR_ARG;
+    if ((c->flags & FP8MLP_GU_FP8) && sc->gu == nullptr) return FP8MLP_ERR_ARG;
     if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX && (am == nullptr || am->dy == nullptr || am->dz == nullptr)) return FP8MLP_ERR_ARG;
     if (!aligned16(dy) || !aligned16(dx) || !aligned16(dW1) || !aligned16(dW2) || !aligned16(dW3)) return FP8MLP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -607,6 +620,7 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
         }
         a.s_h = sc->h; a.smooth = smooth ? 1 : 0;
         a.gu = c->gu; a.sdz = sc->dz; a.dzq = c->dzq;
+        if (c->flags & FP8MLP_GU_FP8) { a.gu8 = reinterpret_cast<uint8_t*>(c->gu); a.gu = nullptr; a.s_gu = sc->gu; }
         a.amax_dz = reinterpret_cast<unsigned int*>(a_dz);
         if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX) {
             a.store = 0;

@@ -199,10 +199,10 @@ __device__ __forceinline__ void store_fp8x32(uint8_t* dst, const float (&v)[32],
 
 // Forward: accumulator columns [0,128) are G = x W2 (gate), [128,256) are U = x W1 (linear) of the
 // same 128 channels; this warp takes channels [64 half, 64 half + 64) of them.
-// H = U * G * sigma(G); per-channel max |H|; Hq = Q_e4m3(H * s_i); bf16 G, U kept for backward.
-// H itself never leaves the SM.
+// H = U * G * sigma(G); per-channel max |H|; Hq = Q_e4m3(H * s_i); G, U kept for backward as bf16, or
+// as E4M3 codes Q(sgu G), Q(sgu U) with their common maximum.  H itself never leaves the SM.
 __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail* tail, uint32_t taddr, int lane,
-                                                    int half, int m, int n0, float dq) {
+                                                    int half, int m, int n0, float dq, float sgu, float& gu_max) {
     const bool row_ok = m < p.M;
     const int f = p.N;
 #pragma unroll 1
@@ -235,9 +235,24 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
             }
             atomicMax(&tail->amax_tile[32 * j + lane], __float_as_uint(colmax));
         }
+        if (p.amax_gu != nullptr) {       // rows past M and columns past f hold zeros
+            float mx = gu_max;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, fmaxf(fabsf(g[e]), fabsf(u[e])));
+            gu_max = mx;
+        }
         if (!p.store || !row_ok) continue;
         const bool both = c0 + 16 < f;
-        if (p.gu != nullptr) {
+        if (p.gu8 != nullptr) {
+            uint8_t* grow = p.gu8 + static_cast<int64_t>(m) * 2 * f + c0;
+            float t[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) t[e] = __fmul_rn(g[e], sgu);
+            store_fp8x32<FP8MLP_E4M3>(grow, t, both, p.wide);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) t[e] = __fmul_rn(u[e], sgu);
+            store_fp8x32<FP8MLP_E4M3>(grow + f, t, both, p.wide);
+        } else if (p.gu != nullptr) {
             uint16_t* grow = p.gu + static_cast<int64_t>(m) * 2 * f + c0;
             store_bf16x16(grow, g, true);
             store_bf16x16(grow + f, u, true);
@@ -262,14 +277,17 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
 // each chunk this warp takes channels [32 half, 32 half + 32).  The saved bf16 G and U of a chunk arrive
 // in shared memory (loader warp, TMA, 128-byte swizzle: the 16-byte piece j of row r sits at piece
 // j ^ (r & 7)); the thread copies its row's 64 + 64 bytes to registers and hands the slot back.
+// Kept as E4M3 codes instead (p.gu8), a slot holds 128 channels of G and of U - two chunks - the thread
+// copies 32 + 32 bytes per chunk, hands the slot back after the second, and G = code * (1 / sgu).
 // dH = acc * dq (* s_i with Smooth-SwiGLU); dU = dH * G sigma(G);
 // dG = dH * U * sigma(G) (1 + G (1 - sigma(G))); max of |dG|, |dU|; dZq = Q_e5m2([dG | dU] * sdz).
 // Returns false if a wait ran out.
 __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail* tail, uint32_t gu_base, uint32_t& gu_count,
                                                     const float* s_tile, uint32_t taddr, int lane, int half, int row,
-                                                    int m, int n0, float dq, float sdz, volatile int* abort_flag,
-                                                    float& run_max) {
+                                                    int m, int n0, float dq, float sdz, float inv_sgu,
+                                                    volatile int* abort_flag, float& run_max) {
     const bool row_ok = m < p.M;
+    const bool gu8 = p.gu8 != nullptr;
     const int f = p.N;
     float local_max = 0.0f;
     // A power-of-two sdz (what fp8mlp_update_scales produces) commutes with every rounding below, so it
@@ -278,23 +296,37 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
     const bool fold = (__float_as_uint(sdz) & 0x007FFFFFu) == 0u && sdz > 1.0e-30f && sdz < 1.0e30f;
     if (fold) dq = __fmul_rn(dq, sdz);
 #pragma unroll 1
-    for (int c = 0; c < 4; ++c, ++gu_count) {
+    for (int c = 0; c < 4; ++c) {
         const uint32_t slot = gu_count % kGuSlots, phase = (gu_count / kGuSlots) & 1u;
         const int col = 64 * c + 32 * half;            // first of this warp's 32 accumulator columns
         const int c0 = n0 + col;
-        if (!mbar_wait(smem_u32(&tail->gu_full[slot]), phase, abort_flag, p.status)) return false;
+        if (!gu8 || (c & 1) == 0)                      // codes: the slot of chunk c - 1 also holds chunk c
+            if (!mbar_wait(smem_u32(&tail->gu_full[slot]), phase, abort_flag, p.status)) return false;
         uint4 gq[4], uq[4];
         {
             const uint32_t rbase = gu_base + slot * kGuSlotBytes + static_cast<uint32_t>(row) * 128u;
+            if (gu8) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t off = static_cast<uint32_t>(((4 * half + i) ^ (row & 7)) * 16);
-                gq[i] = ld_shared_v4(rbase + off);
-                uq[i] = ld_shared_v4(rbase + kBoxBytes + off);
+                for (int i = 0; i < 2; ++i) {
+                    const uint32_t off = static_cast<uint32_t>(((4 * (c & 1) + 2 * half + i) ^ (row & 7)) * 16);
+                    gq[i] = ld_shared_v4(rbase + off);
+                    uq[i] = ld_shared_v4(rbase + kBoxBytes + off);
+                }
+                gq[2] = gq[3] = uq[2] = uq[3] = make_uint4(0u, 0u, 0u, 0u);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t off = static_cast<uint32_t>(((4 * half + i) ^ (row & 7)) * 16);
+                    gq[i] = ld_shared_v4(rbase + off);
+                    uq[i] = ld_shared_v4(rbase + kBoxBytes + off);
+                }
             }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tail->gu_empty[slot]));     // the chunk is in registers
+        if (!gu8 || (c & 1) == 1) {
+            if (lane == 0) mbar_arrive(smem_u32(&tail->gu_empty[slot]));     // the slot's data is in registers
+            ++gu_count;
+        }
         if (c0 >= f) continue;
         uint32_t acc[32];
         tmem_ld32(taddr + col, acc);
@@ -309,7 +341,13 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
         for (int q = 0; q < 16; ++q) {
             dh2[q] = mul2(pack2(__uint_as_float(acc[2 * q]), __uint_as_float(acc[2 * q + 1])), dq2);
             if (p.smooth) dh2[q] = mul2(dh2[q], pack2(s_tile[col + 2 * q], s_tile[col + 2 * q + 1]));
-            g2[q] = pack2(bf16_lo(gw[q]), bf16_hi(gw[q]));
+            if (gu8) {
+                float a, b;
+                e4m3x2_to_f32(gw[q >> 1] >> (16 * (q & 1)), a, b);
+                g2[q] = mul2(pack2(a, b), pack2(inv_sgu, inv_sgu));
+            } else {
+                g2[q] = pack2(bf16_lo(gw[q]), bf16_hi(gw[q]));
+            }
         }
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
@@ -325,7 +363,14 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
         }
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
-            const f32x2 u2 = pack2(bf16_lo(uw[q]), bf16_hi(uw[q]));
+            f32x2 u2;
+            if (gu8) {
+                float a, b;
+                e4m3x2_to_f32(uw[q >> 1] >> (16 * (q & 1)), a, b);
+                u2 = mul2(pack2(a, b), pack2(inv_sgu, inv_sgu));
+            } else {
+                u2 = pack2(bf16_lo(uw[q]), bf16_hi(uw[q]));
+            }
             const f32x2 du_2 = mul2(dh2[q], mul2(g2[q], sig2[q]));
             const f32x2 t1 = add2(one2, mul2(g2[q], sub2(one2, sig2[q])));
             const f32x2 dg_2 = mul2(mul2(dh2[q], u2), mul2(sig2[q], t1));
@@ -498,14 +543,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     tile_coords(p, tile, m_tile, n_tile);
                     const int m0 = m_tile * kTileM + static_cast<int>(rank) * kBlockM;
                     const int n0 = n_tile * p.n_tile_cols;
-                    for (int c = 0; c < 4; ++c, ++count) {
+                    // per slot 64 channels of bf16 G and U, or 128 channels of their E4M3 codes: 4 or 2 slots a tile
+                    const int n_slots = p.gu8 != nullptr ? 2 : 4, per_slot = p.gu8 != nullptr ? 128 : 64;
+                    for (int c = 0; c < n_slots; ++c, ++count) {
                         const uint32_t slot = count % kGuSlots, phase = (count / kGuSlots) & 1u;
                         if (!mbar_wait(smem_u32(&tail->gu_empty[slot]), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
                         const uint32_t bar = smem_u32(&tail->gu_full[slot]);
                         const uint32_t dst = gu_base + slot * kGuSlotBytes;
                         mbar_expect_tx(bar, kGuSlotBytes);
-                        tma_load_2d(dst, &tmG, bar, n0 + 64 * c, m0);              // columns past f read as zeros
-                        tma_load_2d(dst + kBoxBytes, &tmU, bar, n0 + 64 * c, m0);
+                        tma_load_2d(dst, &tmG, bar, n0 + per_slot * c, m0);        // columns past f read as zeros
+                        tma_load_2d(dst + kBoxBytes, &tmU, bar, n0 + per_slot * c, m0);
                     }
                 }
             }
@@ -520,6 +567,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         float sdz = 1.0f;
         if constexpr (EPI == EPI_SWIGLU_BWD) sdz = *p.sdz;
         float run_max = 0.0f;
+        float sgu = 1.0f, inv_sgu = 1.0f, gu_max = 0.0f;     // saved G, U as E4M3 codes: scale, reciprocal, running max
+        if constexpr (EPI == EPI_SWIGLU_FWD || EPI == EPI_SWIGLU_BWD) {
+            if (p.gu8 != nullptr) { sgu = *p.s_gu; inv_sgu = __fdiv_rn(1.0f, sgu); }
+        }
         uint32_t gu_count = 0;                         // chunks of saved G, U consumed so far (backward)
         int it = 0;
         for (int tile = first_tile; tile < num_tiles; tile += tile_step, ++it) {
@@ -549,10 +600,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 epilogue_bf16(p, taddr, half, m, n0, dq0);
                 if constexpr (WIDEN) epilogue_bf16(p, taddr + kBlockN, half, m, n0 + kBlockN, dq0);
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
-                epilogue_swiglu_fwd(p, tail, taddr, lane, half, m, n0, dq0);
+                epilogue_swiglu_fwd(p, tail, taddr, lane, half, m, n0, dq0, sgu, gu_max);
             } else {
                 const bool fine = epilogue_swiglu_bwd(p, tail, gu_base, gu_count, tail->s_tile[acc], taddr, lane, half, row,
-                                                      m, n0, dq0, sdz, abort_flag, run_max);
+                                                      m, n0, dq0, sdz, inv_sgu, abort_flag, run_max);
                 if (!epi_all(fine)) break;
             }
             // accumulator drained: hand it back to the MMA warp (of rank 0)
@@ -575,6 +626,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if constexpr (EPI == EPI_SWIGLU_BWD) {
             run_max = warp_max_nonneg(run_max);
             if (lane == 0 && run_max > 0.0f) atomicMax(p.amax_dz, __float_as_uint(run_max));
+        }
+        if constexpr (EPI == EPI_SWIGLU_FWD) {
+            if (p.amax_gu != nullptr) {
+                gu_max = warp_max_nonneg(gu_max);
+                if (lane == 0 && gu_max > 0.0f) atomicMax(p.amax_gu, __float_as_uint(gu_max));
+            }
         }
     }
 
@@ -621,8 +678,14 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
     CUtensorMap tmG = tmA, tmU = tmA;
     if (EPI == EPI_SWIGLU_BWD) {
         const uint64_t f = static_cast<uint64_t>(args.N), rows = static_cast<uint64_t>(args.M);
-        int rc = make_tmap(&tmG, args.gu, 2, false, f, rows, 4 * f);
-        if (rc == FP8MLP_OK) rc = make_tmap(&tmU, args.gu + f, 2, false, f, rows, 4 * f);
+        int rc;
+        if (args.gu8 != nullptr) {       // E4M3 codes [M, 2f]: boxes of 128 channels
+            rc = make_tmap_u8(&tmG, args.gu8, f, rows, 2 * f);
+            if (rc == FP8MLP_OK) rc = make_tmap_u8(&tmU, args.gu8 + f, f, rows, 2 * f);
+        } else {
+            rc = make_tmap(&tmG, args.gu, 2, false, f, rows, 4 * f);
+            if (rc == FP8MLP_OK) rc = make_tmap(&tmU, args.gu + f, 2, false, f, rows, 4 * f);
+        }
         if (rc != FP8MLP_OK) return rc;
     }
     static std::once_flag once;
@@ -719,7 +782,7 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     switch (epi) {
         case EPI_F32: args.wide = al32(args.out_f32_0) && al32(args.out_f32_1); break;
         case EPI_BF16: args.wide = al32(args.out_bf16); break;
-        case EPI_SWIGLU_FWD: args.wide = al32(args.hq) && args.N % 32 == 0; break;
+        case EPI_SWIGLU_FWD: args.wide = al32(args.hq) && al32(args.gu8) && args.N % 32 == 0; break;
         default: args.wide = al32(args.dzq) && args.N % 32 == 0; break;
     }
     const int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;

@@ -69,6 +69,9 @@ struct GemmArgs {
     uint8_t* hq;            // fwd: E4M3 [M, f]
     uint16_t* hb;           // fwd: if not null, bf16 [M, f] = H unscaled, stored instead of hq (32-byte aligned rows)
     uint16_t* gu;           // fwd: out (nullable), bwd: in; bf16 [M, 2f] = G | U
+    uint8_t* gu8;           // if not null: E4M3 [M, 2f] = Q(s_gu [G | U]) kept instead of the bf16 pair (fwd: out, bwd: in)
+    const float* s_gu;      // scale of gu8
+    unsigned int* amax_gu;  // fwd: bit pattern of max(|G|, |U|), raised atomically; null: not wanted
     unsigned int* amax_h;   // fwd: [f] bit patterns of max |H|, raised atomically; null: maxima not wanted
     const float* sdz;       // bwd: scale of dZ
     uint8_t* dzq;           // bwd: E5M2 [M, 2f] = dG | dU

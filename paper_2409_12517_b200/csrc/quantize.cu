@@ -178,6 +178,7 @@ __global__ void __launch_bounds__(kThreads) update_scales_kernel(UpdateScalesArg
         if (a.amax_w3 && a.scale_w3) *a.scale_w3 = scale_from_amax_dev(FP8MLP_E4M3, *a.amax_w3);
         if (a.amax_dy && a.scale_dy) *a.scale_dy = scale_from_amax_dev(FP8MLP_E5M2, *a.amax_dy);
         if (a.amax_dz && a.scale_dz) *a.scale_dz = pow2_scale_dev(FP8MLP_E5M2, *a.amax_dz);
+        if (a.amax_gu && a.scale_gu) *a.scale_gu = scale_from_amax_dev(FP8MLP_E4M3, *a.amax_gu);
     }
     if (a.amax_h == nullptr || a.scale_h == nullptr) return;
     if (a.smooth) {

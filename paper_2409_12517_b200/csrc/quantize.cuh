@@ -43,8 +43,8 @@ int run_cast_bf16(const float* src, uint16_t* dst, int64_t n, float* amax_out, i
 int run_scale_from_amax(int fmt, const float* amax_a, const float* amax_b, float* scale, cudaStream_t st);
 
 struct UpdateScalesArgs {
-    const float *amax_x, *amax_w1, *amax_w2, *amax_w3, *amax_dy, *amax_dz, *amax_h;
-    float *scale_x, *scale_w12, *scale_w3, *scale_dy, *scale_dz, *scale_h;
+    const float *amax_x, *amax_w1, *amax_w2, *amax_w3, *amax_dy, *amax_dz, *amax_h, *amax_gu;
+    float *scale_x, *scale_w12, *scale_w3, *scale_dy, *scale_dz, *scale_h, *scale_gu;
     int64_t f;
     int smooth;
 };

@@ -272,3 +272,48 @@ def test_7b_forward_just_in_time_scales_sampled_channels():
                          sx=sx, sw12=sw12, s_h=s_ref, sw3=1.0)
     frac, worst = code_mismatch(hq_cols, fwc["Hq"])
     assert worst <= 1 and frac <= CODE_FRAC, f"Hq columns: {frac:.2e} differ, worst {worst}"
+
+
+def test_7b_saved_activations_in_fp8_sampled_tokens():
+    """FP8MLP_GU_FP8 at the benchmark's 7B size (delayed scaling): whole rows of the saved E4M3 codes of G, U and of
+    what backward makes of them (dZq, dX), and the maximum of |G|, |U| against the sample's."""
+    w = wl.make_config("7b")
+    T, d, f = w.T, w.d, w.f
+    given = _previous_iteration_scales(w, 32, True)
+    cfg = dict(wl.CONFIGS[w.name]); cfg.update(seed=cfg["seed"] + 100, T=32)
+    prev = wl.make("prev", **cfg)
+    pf = oracle.forward(prev.x, w.W1, w.W2, w.W3, flags=oracle.FLAG_SMOOTH | oracle.FLAG_GU_FP8)
+    given["gu"] = np.float32(pf["sgu"] * 0.25)
+    rng = np.random.default_rng(4321)
+    toks = _sample(rng, T, 16, w.outlier_tokens[:4])
+    ctx = B.fp8mlp_create(T, d, f, B.SMOOTH | B.SAVE_FOR_BWD | B.GU_FP8)
+    try:
+        sc, am = B.new_scales(f), B.new_amax(f)
+        for k, v in given.items():
+            sc[k].copy_(to_dev(np.atleast_1d(np.asarray(v, np.float32))))
+        W1, W2, W3 = to_dev(w.W1), to_dev(w.W2), to_dev(w.W3)
+        y = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        dx = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        dW1, dW2, dW3 = torch.empty((d, f), device="cuda"), torch.empty((d, f), device="cuda"), torch.empty((f, d), device="cuda")
+        B.fp8mlp_forward(ctx, T, to_dev_bf16(w.x), W1, W2, W3, B.SCALE_GIVEN, sc, am, y)
+        B.fp8mlp_backward(ctx, T, to_dev_bf16(w.dY), B.SCALE_GIVEN, sc, am, dx, dW1, dW2, dW3)
+        assert B.fp8mlp_status(ctx) == B.OK
+        ti = torch.from_numpy(toks).cuda()
+        gu_rows = B.workspace_tensor(ctx, B.WS_GU, (T, 2 * f), torch.uint8)[ti].cpu().numpy()
+        dz_rows = B.workspace_tensor(ctx, B.WS_DZQ, (T, 2 * f), torch.uint8)[ti].cpu().numpy()
+        dx_rows = dx[ti].view(torch.int16).cpu().numpy().view(np.uint16)
+        a_gu, s_gu = am["gu"].item(), sc["gu"].item()
+    finally:
+        B.fp8mlp_destroy(ctx)
+    assert s_gu == given["gu"]
+    fw = oracle.forward(w.x[toks], w.W1, w.W2, w.W3, flags=oracle.FLAG_SMOOTH | oracle.FLAG_GU_FP8,
+                        scale_mode=oracle.SCALE_GIVEN, sx=float(given["x"]), sw12=float(given["w12"]), s_h=given["h"],
+                        sw3=float(given["w3"]), sgu=float(given["gu"]))
+    bw = oracle.backward(fw, w.dY[toks], scale_mode=oracle.SCALE_GIVEN, sdy=float(given["dy"]), sdz=float(given["dz"]))
+    assert a_gu >= 0.99999 * fw["amax_gu"]                   # the global maximum covers the sample's
+    frac, worst = code_mismatch(gu_rows, fw["GUq"])
+    assert worst <= 1 and frac <= CODE_FRAC, f"saved G, U codes: {frac:.2e} differ, worst {worst}"
+    _check_dz_codes("dZq rows", dz_rows, bw["dZq"])
+    inv = lambda v: np.float32(1.0) / np.float32(v)
+    dx_shift = _explained(oracle.E5M2, dz_rows, bw["dZq"], fw["W12q"], False, inv(given["dz"]) * inv(given["w12"]))
+    _check_bf16_rows("dX", dx_rows, bw["dX"] + dx_shift)
