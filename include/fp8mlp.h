@@ -46,7 +46,8 @@ enum {
     FP8MLP_ERR_ALIGN = -3,   /* a tensor pointer is not 16-byte aligned                         */
     FP8MLP_ERR_CUDA = -4,    /* a CUDA runtime/driver call failed (see fp8mlp_last_cuda_error)  */
     FP8MLP_ERR_TIMEOUT = -5, /* a kernel gave up on a bounded wait (device status word)         */
-    FP8MLP_ERR_STATE = -6,   /* backward without a matching forward that saved activations      */
+    FP8MLP_ERR_STATE = -6,   /* backward without a matching forward that saved activations; merged forward
+                                without merged weights; the context's device is not the current one */
     FP8MLP_ERR_TOO_LARGE = -7 /* fp8mlp_forward_static: the problem does not fit the built-in scratch */
 };
 enum { FP8MLP_E4M3 = 0, FP8MLP_E5M2 = 1 };

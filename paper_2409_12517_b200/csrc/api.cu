@@ -97,6 +97,13 @@ struct PhaseTimer {
     }
 };
 
+// A context's buffers live on the device that was current when it was created: calls on it must be
+// made with that device current.
+bool on_device_of(const fp8mlp_ctx* c) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == c->device;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int zero_floats(std::initializer_list<float*> ptrs, cudaStream_t st, float* vec = nullptr, int64_t n_vec = 0) {
@@ -203,7 +210,8 @@ const char* fp8mlp_strerror(int code) {
         case FP8MLP_ERR_ALIGN: return "pointer not 16-byte aligned";
         case FP8MLP_ERR_CUDA: return "CUDA call failed";
         case FP8MLP_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
-        case FP8MLP_ERR_STATE: return "backward without a matching forward that saved activations";
+        case FP8MLP_ERR_STATE: return "call does not fit the context's state (backward without a matching forward that saved "
+                                      "activations, merged forward without merged weights, or another device is current)";
         case FP8MLP_ERR_TOO_LARGE: return "problem does not fit the library's built-in scratch (see FP8MLP_STATIC_SCRATCH_BYTES)";
         default: return "unknown error code";
     }
@@ -379,6 +387,7 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
                    int mode, fp8mlp_scales* sc, fp8mlp_amax* am, void* y, void* stream) {
     if (c == nullptr || sc == nullptr || W1 == nullptr || W2 == nullptr || W3 == nullptr) return FP8MLP_ERR_ARG;
     if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
+    if (!on_device_of(c)) return FP8MLP_ERR_STATE;
     if (T < 0 || T > c->T_max) return FP8MLP_ERR_SHAPE;
     if (T > 0 && (x == nullptr || y == nullptr)) return FP8MLP_ERR_ARG;
     if (sc->x == nullptr || sc->w12 == nullptr || sc->w3 == nullptr || sc->h == nullptr) return FP8MLP_ERR_ARG;
@@ -493,6 +502,7 @@ int fp8mlp_merge_weights(fp8mlp_ctx* c, const float* W1, const float* W2, const 
     if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
     if (sc->w12 == nullptr || sc->w3 == nullptr) return FP8MLP_ERR_ARG;
     if (c->flags & FP8MLP_H_BF16) return FP8MLP_ERR_STATE;          // this context has no FP8 W3
+    if (!on_device_of(c)) return FP8MLP_ERR_STATE;
     if (!aligned16(W1) || !aligned16(W2) || !aligned16(W3) || !aligned16(s)) return FP8MLP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t d = c->d, f = c->f;
@@ -525,7 +535,7 @@ int fp8mlp_forward_merged(fp8mlp_ctx* c, int64_t T, const void* x, int mode, fp8
     if (c == nullptr || sc == nullptr) return FP8MLP_ERR_ARG;
     if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
     if (T < 0 || T > c->T_max) return FP8MLP_ERR_SHAPE;
-    if (!c->merged) return FP8MLP_ERR_STATE;
+    if (!on_device_of(c) || !c->merged) return FP8MLP_ERR_STATE;
     if (T > 0 && (x == nullptr || y == nullptr)) return FP8MLP_ERR_ARG;
     if (sc->x == nullptr || sc->w12 == nullptr || sc->w3 == nullptr || sc->h == nullptr) return FP8MLP_ERR_ARG;
     if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX && (am == nullptr || am->x == nullptr || am->h == nullptr)) return FP8MLP_ERR_ARG;
@@ -573,6 +583,7 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
     if (c == nullptr || sc == nullptr || dW1 == nullptr || dW2 == nullptr || dW3 == nullptr) return FP8MLP_ERR_ARG;
     if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
     if (T < 0 || T > c->T_max) return FP8MLP_ERR_SHAPE;
+    if (!on_device_of(c)) return FP8MLP_ERR_STATE;
     if (!(c->flags & FP8MLP_SAVE_FOR_BWD) || c->saved_T != T) return FP8MLP_ERR_STATE;
     if (T > 0 && (dy == nullptr || dx == nullptr)) return FP8MLP_ERR_ARG;
     if (sc->x == nullptr || sc->w12 == nullptr || sc->w3 == nullptr || sc->h == nullptr || sc->dy == nullptr || sc->dz == nullptr)

@@ -200,7 +200,8 @@ __device__ __forceinline__ void store_fp8x32(uint8_t* dst, const float (&v)[32],
 // Forward: accumulator columns [0,128) are G = x W2 (gate), [128,256) are U = x W1 (linear) of the
 // same 128 channels; this warp takes channels [64 half, 64 half + 64) of them.
 // H = U * G * sigma(G); per-channel max |H|; Hq = Q_e4m3(H * s_i); G, U kept for backward as bf16, or
-// as E4M3 codes Q(sgu G), Q(sgu U) with their common maximum.  H itself never leaves the SM.
+// as E4M3 codes Q(sgu G), Q(sgu U) with their common maximum (GU8).  H itself never leaves the SM.
+template <bool GU8>
 __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail* tail, uint32_t taddr, int lane,
                                                     int half, int m, int n0, float dq, float sgu, float& gu_max) {
     const bool row_ok = m < p.M;
@@ -235,7 +236,7 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
             }
             atomicMax(&tail->amax_tile[32 * j + lane], __float_as_uint(colmax));
         }
-        if (p.amax_gu != nullptr) {       // rows past M and columns past f hold zeros
+        if constexpr (GU8) {              // rows past M and columns past f hold zeros
             float mx = gu_max;
 #pragma unroll
             for (int e = 0; e < 32; ++e) mx = fmaxf(mx, fmaxf(fabsf(g[e]), fabsf(u[e])));
@@ -243,7 +244,7 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
         }
         if (!p.store || !row_ok) continue;
         const bool both = c0 + 16 < f;
-        if (p.gu8 != nullptr) {
+        if constexpr (GU8) {
             uint8_t* grow = p.gu8 + static_cast<int64_t>(m) * 2 * f + c0;
             float t[32];
 #pragma unroll
@@ -252,7 +253,8 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
 #pragma unroll
             for (int e = 0; e < 32; ++e) t[e] = __fmul_rn(u[e], sgu);
             store_fp8x32<FP8MLP_E4M3>(grow + f, t, both, p.wide);
-        } else if (p.gu != nullptr) {
+        }
+        if (!GU8 && p.gu != nullptr) {
             uint16_t* grow = p.gu + static_cast<int64_t>(m) * 2 * f + c0;
             store_bf16x16(grow, g, true);
             store_bf16x16(grow + f, u, true);
@@ -281,13 +283,14 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
 // copies 32 + 32 bytes per chunk, hands the slot back after the second, and G = code * (1 / sgu).
 // dH = acc * dq (* s_i with Smooth-SwiGLU); dU = dH * G sigma(G);
 // dG = dH * U * sigma(G) (1 + G (1 - sigma(G))); max of |dG|, |dU|; dZq = Q_e5m2([dG | dU] * sdz).
-// Returns false if a wait ran out.
+// Returns false if a wait ran out.  GU8: the saved activations are E4M3 codes (p.gu8), else bf16 (p.gu).
+template <bool GU8>
 __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail* tail, uint32_t gu_base, uint32_t& gu_count,
                                                     const float* s_tile, uint32_t taddr, int lane, int half, int row,
                                                     int m, int n0, float dq, float sdz, float inv_sgu,
                                                     volatile int* abort_flag, float& run_max) {
     const bool row_ok = m < p.M;
-    const bool gu8 = p.gu8 != nullptr;
+    constexpr bool gu8 = GU8;
     const int f = p.N;
     float local_max = 0.0f;
     // A power-of-two sdz (what fp8mlp_update_scales produces) commutes with every rounding below, so it
@@ -305,7 +308,7 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
         uint4 gq[4], uq[4];
         {
             const uint32_t rbase = gu_base + slot * kGuSlotBytes + static_cast<uint32_t>(row) * 128u;
-            if (gu8) {
+            if constexpr (gu8) {
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
                     const uint32_t off = static_cast<uint32_t>(((4 * (c & 1) + 2 * half + i) ^ (row & 7)) * 16);
@@ -341,7 +344,7 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
         for (int q = 0; q < 16; ++q) {
             dh2[q] = mul2(pack2(__uint_as_float(acc[2 * q]), __uint_as_float(acc[2 * q + 1])), dq2);
             if (p.smooth) dh2[q] = mul2(dh2[q], pack2(s_tile[col + 2 * q], s_tile[col + 2 * q + 1]));
-            if (gu8) {
+            if constexpr (gu8) {
                 float a, b;
                 e4m3x2_to_f32(gw[q >> 1] >> (16 * (q & 1)), a, b);
                 g2[q] = mul2(pack2(a, b), pack2(inv_sgu, inv_sgu));
@@ -364,7 +367,7 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             f32x2 u2;
-            if (gu8) {
+            if constexpr (gu8) {
                 float a, b;
                 e4m3x2_to_f32(uw[q >> 1] >> (16 * (q & 1)), a, b);
                 u2 = mul2(pack2(a, b), pack2(inv_sgu, inv_sgu));
@@ -401,7 +404,8 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
 // PAIR = false: one CTA per 128 x 256 tile.  PAIR = true: a cluster of two CTAs per 256 x 256 tile
 // (tcgen05 cta_group::2): rank r loads rows [128 r, 128 r + 128) of the A tile and of the B tile,
 // rank 0 issues the MMAs for both, and each CTA drains its own 128 rows of the accumulator.
-template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM, bool WIDEN>
+// GU8 (SwiGLU epilogues only): the activations saved for backward are E4M3 codes (args.gu8), not bf16.
+template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM, bool WIDEN, bool GU8>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
             const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmG,
@@ -410,6 +414,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     constexpr int kStageBytes = Plan<PAIR, EPI, WIDEN>::kStageBytes;
     constexpr int kTileM = Plan<PAIR, EPI, WIDEN>::kTileM;
     static_assert(!WIDEN || (PAIR && (EPI == EPI_F32 || EPI == EPI_BF16)), "wide tiles: CTA pairs, plain epilogues");
+    static_assert(!GU8 || EPI == EPI_SWIGLU_BWD || EPI == EPI_SWIGLU_FWD, "GU8 belongs to the SwiGLU epilogues");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;         // swizzle atoms need 1024-byte alignment
@@ -544,7 +549,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     const int m0 = m_tile * kTileM + static_cast<int>(rank) * kBlockM;
                     const int n0 = n_tile * p.n_tile_cols;
                     // per slot 64 channels of bf16 G and U, or 128 channels of their E4M3 codes: 4 or 2 slots a tile
-                    const int n_slots = p.gu8 != nullptr ? 2 : 4, per_slot = p.gu8 != nullptr ? 128 : 64;
+                    constexpr int n_slots = GU8 ? 2 : 4, per_slot = GU8 ? 128 : 64;
                     for (int c = 0; c < n_slots; ++c, ++count) {
                         const uint32_t slot = count % kGuSlots, phase = (count / kGuSlots) & 1u;
                         if (!mbar_wait(smem_u32(&tail->gu_empty[slot]), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
@@ -569,7 +574,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         float run_max = 0.0f;
         float sgu = 1.0f, inv_sgu = 1.0f, gu_max = 0.0f;     // saved G, U as E4M3 codes: scale, reciprocal, running max
         if constexpr (EPI == EPI_SWIGLU_FWD || EPI == EPI_SWIGLU_BWD) {
-            if (p.gu8 != nullptr) { sgu = *p.s_gu; inv_sgu = __fdiv_rn(1.0f, sgu); }
+            if constexpr (GU8) { sgu = *p.s_gu; inv_sgu = __fdiv_rn(1.0f, sgu); }
         }
         uint32_t gu_count = 0;                         // chunks of saved G, U consumed so far (backward)
         int it = 0;
@@ -600,10 +605,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 epilogue_bf16(p, taddr, half, m, n0, dq0);
                 if constexpr (WIDEN) epilogue_bf16(p, taddr + kBlockN, half, m, n0 + kBlockN, dq0);
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
-                epilogue_swiglu_fwd(p, tail, taddr, lane, half, m, n0, dq0, sgu, gu_max);
+                epilogue_swiglu_fwd<GU8>(p, tail, taddr, lane, half, m, n0, dq0, sgu, gu_max);
             } else {
-                const bool fine = epilogue_swiglu_bwd(p, tail, gu_base, gu_count, tail->s_tile[acc], taddr, lane, half, row,
-                                                      m, n0, dq0, sdz, inv_sgu, abort_flag, run_max);
+                const bool fine = epilogue_swiglu_bwd<GU8>(p, tail, gu_base, gu_count, tail->s_tile[acc], taddr, lane, half, row,
+                                                           m, n0, dq0, sdz, inv_sgu, abort_flag, run_max);
                 if (!epi_all(fine)) break;
             }
             // accumulator drained: hand it back to the MMA warp (of rank 0)
@@ -627,11 +632,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             run_max = warp_max_nonneg(run_max);
             if (lane == 0 && run_max > 0.0f) atomicMax(p.amax_dz, __float_as_uint(run_max));
         }
-        if constexpr (EPI == EPI_SWIGLU_FWD) {
-            if (p.amax_gu != nullptr) {
-                gu_max = warp_max_nonneg(gu_max);
-                if (lane == 0 && gu_max > 0.0f) atomicMax(p.amax_gu, __float_as_uint(gu_max));
-            }
+        if constexpr (EPI == EPI_SWIGLU_FWD && GU8) {
+            gu_max = warp_max_nonneg(gu_max);
+            if (lane == 0 && gu_max > 0.0f) atomicMax(p.amax_gu, __float_as_uint(gu_max));
         }
     }
 
@@ -670,16 +673,16 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM, bool WIDEN = false>
+template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM, bool WIDEN = false, bool GU8 = false>
 int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorMap& tmB1, const GemmArgs& args,
                 int64_t tiles, int sm_count, cudaStream_t st) {
     constexpr size_t kSmem = smem_bytes<PAIR, EPI, WIDEN>();
     // the saved activations [M, 2f] bf16 as two matrices of f columns: G, and U starting f elements in
     CUtensorMap tmG = tmA, tmU = tmA;
-    if (EPI == EPI_SWIGLU_BWD) {
+    if constexpr (EPI == EPI_SWIGLU_BWD) {
         const uint64_t f = static_cast<uint64_t>(args.N), rows = static_cast<uint64_t>(args.M);
         int rc;
-        if (args.gu8 != nullptr) {       // E4M3 codes [M, 2f]: boxes of 128 channels
+        if (GU8) {                       // E4M3 codes [M, 2f]: boxes of 128 channels
             rc = make_tmap_u8(&tmG, args.gu8, f, rows, 2 * f);
             if (rc == FP8MLP_OK) rc = make_tmap_u8(&tmU, args.gu8 + f, f, rows, 2 * f);
         } else {
@@ -688,9 +691,17 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
         }
         if (rc != FP8MLP_OK) return rc;
     }
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    static int max_clusters = 0;
+    // the function attribute and the occupancy answer belong to a device: looked up once per device
+    constexpr int kMaxDevices = 64;
+    static std::once_flag once_dev[kMaxDevices];
+    static cudaError_t attr_err_dev[kMaxDevices] = {};
+    static int max_clusters_dev[kMaxDevices] = {};
+    int dev = 0;
+    FP8MLP_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) { set_cuda_error_str("gemm launch", "device ordinal out of range"); return FP8MLP_ERR_CUDA; }
+    std::once_flag& once = once_dev[dev];
+    cudaError_t& attr_err = attr_err_dev[dev];
+    int& max_clusters = max_clusters_dev[dev];
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     cfg.blockDim = dim3(kGemmThreads);
@@ -705,12 +716,12 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
         cfg.numAttrs = 1;
     }
     std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN, GU8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(kSmem));
         if (PAIR && attr_err == cudaSuccess) {
             // how many CTA pairs the device can hold at once (one CTA per SM, pairs on neighbouring SMs)
             cfg.gridDim = dim3(static_cast<unsigned>(sm_count) & ~1u);
-            attr_err = cudaOccupancyMaxActiveClusters(&max_clusters, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN>, &cfg);
+            attr_err = cudaOccupancyMaxActiveClusters(&max_clusters, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN, GU8>, &cfg);
         }
     });
     FP8MLP_CUDA_CHECK(attr_err);
@@ -722,7 +733,7 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
         grid = tiles < sm_count ? tiles : sm_count;
     }
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
-    FP8MLP_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN>, tmA, tmB0, tmB1, tmG, tmU, args));
+    FP8MLP_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN, GU8>, tmA, tmB0, tmB1, tmG, tmU, args));
     count_launch();
     return FP8MLP_OK;
 }
@@ -808,7 +819,16 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     FP8MLP_DISPATCH(EPI_F32, true, true, 1)
     FP8MLP_DISPATCH(EPI_BF16, false, false, 1)
     FP8MLP_DISPATCH(EPI_BF16, false, true, 1)
+    if (epi == EPI_SWIGLU_FWD && args.gu8 != nullptr) {       // activations kept as E4M3 codes
+        if (a_mn || !b_mn || elem != 1 || args.amax_gu == nullptr || args.s_gu == nullptr) return FP8MLP_ERR_ARG;
+        return pair ? launch_inst<EPI_SWIGLU_FWD, false, true, true, 1, false, true>(tmA, tmB0, tmB1, args, tiles, sm_count, st)
+                    : launch_inst<EPI_SWIGLU_FWD, false, true, false, 1, false, true>(tmA, tmB0, tmB1, args, tiles, sm_count, st);
+    }
     FP8MLP_DISPATCH(EPI_SWIGLU_FWD, false, true, 1)
+    if (epi == EPI_SWIGLU_BWD && args.gu8 != nullptr && (a_mn || b_mn || elem != 1)) return FP8MLP_ERR_ARG;
+    if (epi == EPI_SWIGLU_BWD && args.gu8 != nullptr)      // saved activations as E4M3 codes
+        return pair ? launch_inst<EPI_SWIGLU_BWD, false, false, true, 1, false, true>(tmA, tmB0, tmB1, args, tiles, sm_count, st)
+                    : launch_inst<EPI_SWIGLU_BWD, false, false, false, 1, false, true>(tmA, tmB0, tmB1, args, tiles, sm_count, st);
     FP8MLP_DISPATCH(EPI_SWIGLU_BWD, false, false, 1)
     // the bf16 last layer of the "SwiGLU output in BF16" variant
     FP8MLP_DISPATCH(EPI_BF16, false, true, 2)
