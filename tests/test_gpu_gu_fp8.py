@@ -123,3 +123,28 @@ def test_gu_fp8_flag_combinations():
     h = C.c_void_p()
     assert L.fp8mlp_create(C.byref(h), 16, 16, 16, B.GU_FP8) == B.ERR_ARG                       # nothing is saved
     assert L.fp8mlp_create(C.byref(h), 16, 16, 16, B.GU_FP8 | B.SAVE_FOR_BWD | B.H_BF16) == B.ERR_ARG
+
+
+def test_gu_fp8_empty_batch_and_missing_scale():
+    f = 64
+    w = wl.make("e", 2, 16, 64, f, w_std=0.05)
+    ctx = B.fp8mlp_create(16, 64, f, B.SMOOTH | B.SAVE_FOR_BWD | B.GU_FP8)
+    try:
+        sc, am = B.new_scales(f), B.new_amax(f)
+        W1, W2, W3 = to_dev(w.W1), to_dev(w.W2), to_dev(w.W3)
+        am["gu"].fill_(9.0)
+        B.fp8mlp_forward(ctx, 0, None, W1, W2, W3, B.SCALE_FROM_CURRENT_AMAX, sc, am, None)
+        g = [torch.full((64, 64), 7.0, device="cuda") for _ in range(3)]
+        B.fp8mlp_backward(ctx, 0, None, B.SCALE_FROM_CURRENT_AMAX, sc, am, None, g[0], g[1], g[2])
+        torch.cuda.synchronize()
+        assert am["gu"].item() == 0 and sc["gu"].item() == 1.0      # no tokens: maximum 0, scale falls back to 1
+        assert all(float(t.abs().max()) == 0 for t in g)
+        # a scales struct without the member is refused before anything is launched
+        sc_missing = dict(sc, gu=None)
+        y = torch.zeros((16, 64), dtype=torch.bfloat16, device="cuda")
+        with pytest.raises(B.Fp8MlpError) as ei:
+            B.fp8mlp_forward(ctx, 16, to_dev_bf16(w.x), W1, W2, W3, B.SCALE_GIVEN, sc_missing, am, y)
+        assert ei.value.code == B.ERR_ARG
+        assert B.fp8mlp_status(ctx) == B.OK
+    finally:
+        B.fp8mlp_destroy(ctx)
