@@ -136,7 +136,7 @@ def time_oracle(w, T_s: int, f_s: int):
 def cpu_baseline(w, seconds_target: float = 20.0):
     import oracle
     cores = oracle.num_threads()
-    T_s = min(w.T, max(4, 4 * cores))                 # sized for 10-20 s of host time
+    T_s = min(w.T, max(8, 8 * cores))                 # sized for 10-20 s of host time
     f_s = w.f
     dt = time_oracle(w, T_s, f_s)
     return {"value": flops_step(T_s, w.d, f_s) / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
