@@ -246,6 +246,35 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     ms_step = max_over_ranks(ms_total, world, "cuda") / args.steps
     value = job_tflops(T, d, f, world, ms_step)
 
+    # The same kernels with a fresh power budget: single steps, each after a second of idle, so the board has not
+    # yet throttled.  Context for the sustained figures above (which are what the metric is): not part of value.
+    after_idle = None
+    if rank == 0 and not args.no_after_idle:
+        tdf0 = float(T) * d * f
+        gemm_flops = {"gemm1_swiglu": 4 * tdf0, "gemm2_down": 2 * tdf0, "dgrad2_swiglu_bwd": 2 * tdf0,
+                      "wgrad3": 2 * tdf0, "dgrad1": 4 * tdf0, "wgrad12": 4 * tdf0}
+        best = {k: float("inf") for k in gemm_flops}
+        best_step = float("inf")
+        B.fp8mlp_profile_enable(ctx, True)
+        for _ in range(4):
+            torch.cuda.synchronize()
+            time.sleep(1.0)
+            B.fp8mlp_profile_read(ctx)
+            e0.record()
+            step()
+            e1.record()
+            torch.cuda.synchronize()
+            best_step = min(best_step, e0.elapsed_time(e1))
+            for k, (ms, cnt) in B.fp8mlp_profile_read(ctx).items():
+                if k in best and cnt:
+                    best[k] = min(best[k], ms / cnt)
+        B.fp8mlp_profile_enable(ctx, False)
+        after_idle = {"step_ms": round(best_step, 4), "step_tflops": round(job_tflops(T, d, f, 1, best_step), 1),
+                      "gemm_tflops": {k: round(gemm_flops[k] / (v * 1e-3) / 1e12, 1) for k, v in best.items()},
+                      "gemm_frac_of_nominal_fp8_4500": {k: round(gemm_flops[k] / (v * 1e-3) / 1e12 / NOMINAL_FP8_TFLOPS, 3)
+                                                        for k, v in best.items()},
+                      "what": "best of 4 single steps, each after 1 s of idle (the power cap has not bitten yet)"}
+
     # end to end: inputs start in pinned host memory, results end in host memory, every step
     xh, dyh = x.cpu().pin_memory(), dy.cpu().pin_memory()
     yh, dxh = torch.empty_like(xh).pin_memory(), torch.empty_like(xh).pin_memory()
@@ -445,6 +474,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                                   "step_with_smooth_swiglu_off": plain,
                                   "step_with_swiglu_output_in_bf16": hbf16,
                                   "step_with_saved_activations_in_fp8": gu8,
+                                  "single_step_after_idle": after_idle,
                                   "note": "Adam with E4M3/E5M2 moments on W1, W2, W3, and the inference form of "
                                           "Smooth-SwiGLU; the same step with plain per-tensor FP8 and with the last layer in "
                                           "bf16 (the other rows of the paper's throughput table); the Smooth-SwiGLU step with G, U kept for "
@@ -462,6 +492,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-after-idle", action="store_true", help="skip the single steps timed after a second of idle")
     ap.add_argument("--ref-seconds", type=float, default=120.0,
                     help="--impl reference: CPU time the whole run may take (sizes the channel sample)")
     args = ap.parse_args()
