@@ -70,3 +70,24 @@ def test_binding_refuses_to_run_without_the_library(tmp_path, monkeypatch):
     monkeypatch.setattr(B, "LIB_PATH", tmp_path / "libfp8mlp.so")
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         B.lib()
+
+
+def test_binding_constants_match_the_header():
+    """The Python binding repeats the header's enumerators by value; a drift between the two would pass
+    wrong flags silently."""
+    import ctypes as C
+    header = (ROOT / "include" / "fp8mlp.h").read_text()
+    enums = {name: int(val) for name, val in re.findall(r"\bFP8MLP_([A-Z0-9_]+)\s*=\s*(-?\d+)", header)}
+    for name in ("OK", "ERR_ARG", "ERR_SHAPE", "ERR_ALIGN", "ERR_CUDA", "ERR_TIMEOUT", "ERR_STATE", "E4M3", "E5M2", "BF16", "F32",
+                 "SMOOTH", "SAVE_FOR_BWD", "H_BF16", "GU_FP8", "SCALE_GIVEN", "SCALE_FROM_CURRENT_AMAX",
+                 "WS_XQ", "WS_W12Q", "WS_W3Q", "WS_HQ", "WS_GU", "WS_DYQ", "WS_DZQ", "WS_HB", "WS_W3B"):
+        assert name in enums, name
+        assert getattr(B, name) == enums[name], name
+    phases = [n for n, _ in sorted(((n[3:], v) for n, v in enums.items() if n.startswith("PH_") and n != "PH_COUNT"),
+                                   key=lambda t: t[1])]
+    assert len(B.PHASES) == enums["PH_COUNT"] == len(phases)
+    # the scale / amax structs: one device pointer per member, in the header's order
+    members = lambda typ: re.search(r"typedef struct \{ float ([^}]*); \} " + typ, header).group(1).replace("*", "").replace(" ", "").split(",")
+    assert [n for n, _ in B._Scales._fields_] == members("fp8mlp_scales")
+    assert [n for n, _ in B._Amax._fields_] == members("fp8mlp_amax")
+    assert C.sizeof(B._Scales) == 8 * len(B._Scales._fields_)
