@@ -145,22 +145,28 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One poll of the barrier.  The hardware may park the thread until the phase completes or the hint
+// (nanoseconds) runs out, whichever comes first; without a hint the limit is so short that the waiting
+// warps - eight epilogue warps wait through most of a tile's main loop - keep re-issuing the poll and
+// take issue slots and power from the tensor pipe (GEMM-1 ran 7 % slower that way).
+constexpr uint32_t kSuspendHintNs = 1000000u;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t"
         ".reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t"
         "}\n"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok != 0;
 }
 
 // Bounded wait.  Returns false if the CTA is aborting or the wait ran out of time, in which case
 // it raises the CTA's abort flag (shared) and the global status word; the caller leaves its loop.
+// A poll lasts at most kSuspendHintNs, so the abort flag and the clock are looked at every few of them.
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // 2 s: far beyond any kernel of this library
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort, int* status,
                                           uint64_t timeout_ns = kWaitTimeoutNs) {
@@ -168,7 +174,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     const uint64_t t0 = global_timer_ns();
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63u) == 0u) {
+        if ((spin & 7u) == 0u) {
             if (*cta_abort) return false;
             if (global_timer_ns() - t0 > timeout_ns) {
                 *cta_abort = 1;
