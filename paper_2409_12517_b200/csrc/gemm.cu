@@ -776,7 +776,9 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     // fp32-output weight gradients keep 256 x 256 tiles: their epilogue (four times the bytes) would sit in the open
     // and their tile counts divide worse over the CTA pairs; measured slower with wide tiles.
     const bool widen = pair && args.elem_bytes != 2 && ((epi == EPI_BF16 && args.wide_tiles != 2) || (epi == EPI_F32 && args.wide_tiles == 1)) &&
-                       args.n_tile_cols == kBlockN && args.N >= 2 * kBlockN;
+                       args.n_tile_cols == kBlockN && args.N >= 2 * kBlockN &&
+                       // a small problem needs its tiles for parallelism first: wide tiles only if they still fill the CTA pairs
+                       static_cast<int64_t>(args.num_m_tiles) * ((args.N + 2 * kBlockN - 1) / (2 * kBlockN)) >= sm_count / 2;
     if (widen) args.n_tile_cols = 2 * kBlockN;
     args.num_n_tiles = (args.N + args.n_tile_cols - 1) / args.n_tile_cols;
     const int elem = args.elem_bytes == 2 ? 2 : 1;

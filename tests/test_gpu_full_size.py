@@ -19,7 +19,8 @@ import pytest
 import torch
 
 import oracle
-from helpers import bf16_bits_to_f32, code_mismatch, frac_beyond, nmax_err, nmax_err_bf16, to_dev, to_dev_bf16
+from helpers import (bf16_bits_to_f32, check_dz_codes as _check_dz_codes, code_mismatch, frac_beyond, nmax_err, nmax_err_bf16,
+                     to_dev, to_dev_bf16)
 from paper_2409_12517_b200 import binding as B
 from paper_2409_12517_b200 import workloads as wl
 
@@ -67,23 +68,6 @@ def _explained(code_fmt, got_codes, ref_codes, operand_codes, operand_is_kn, dq)
         return 0.0
     other = operand_codes[idx, :] if operand_is_kn else operand_codes[:, idx].T          # [len(idx), N]
     return (diff[:, idx] @ oracle.decode(oracle.E4M3, np.ascontiguousarray(other)).astype(np.float64)) * float(dq)
-
-
-def _check_dz_codes(name, got, ref):
-    """E5M2 codes of [dG | dU].  They inherit the accumulation-order differences like Hq does (one
-    code step, rarely), and one more: the saved bf16 G and U may themselves differ by one bf16
-    spacing between the two sides, and near the zero of the gate derivative (G about -1.28) that
-    moves a small dG by more than one of its own code steps.  So: few codes differ at all, hardly
-    any by more than one step, and every difference is small against the tensor (the bar for
-    gradient values)."""
-    frac, worst = code_mismatch(got, ref)
-    assert frac <= CODE_FRAC, f"{name}: {frac:.2e} of the codes differ"
-    if worst > 1:
-        from helpers import code_rank
-        many = float(np.mean(np.abs(code_rank(got) - code_rank(ref)) > 1))
-        assert many <= 2e-5, f"{name}: {many:.2e} of the codes differ by more than one step"
-        dv, rv = oracle.decode(oracle.E5M2, got), oracle.decode(oracle.E5M2, ref)
-        assert nmax_err(dv, rv) <= OUT_TOL, f"{name}: decoded difference {nmax_err(dv, rv)}"
 
 
 def _sample(rng, n, count, always=()):

@@ -9,7 +9,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import bf16_dev_to_bits, bf16_bits_to_f32, code_mismatch, nmax_err, to_dev, to_dev_bf16
+from helpers import bf16_dev_to_bits, bf16_bits_to_f32, check_dz_codes, code_mismatch, nmax_err, to_dev, to_dev_bf16
 from paper_2409_12517_b200 import binding as B
 from paper_2409_12517_b200 import workloads as wl
 
@@ -83,13 +83,16 @@ def check_forward(r: Run, fw: dict, save=True):
     assert e <= OUT_TOL, f"Y: {e}"
 
 
-def check_backward(r: Run, bw: dict):
+def check_backward(r: Run, bw: dict, many_codes: bool = False):
     assert r.amax["dy"][0] == np.float32(bw["amax_dy"]) and r.scales["dy"][0] == np.float32(bw["sdy"])
     assert np.array_equal(r.dYq, bw["dYq"]), "dY codes differ"
     assert np.isclose(r.amax["dz"][0], bw["amax_dz"], rtol=1e-3), "amax of dZ"
     assert r.scales["dz"][0] == np.float32(bw["sdz"]), "scale of dZ"
-    frac, worst = code_mismatch(r.dZq, bw["dZq"])
-    assert worst <= 1 and frac <= CODE_FRAC, f"dZq codes: {frac:.2e} differ, worst {worst} steps"
+    if many_codes:      # among hundreds of thousands of codes a few sit at the zero of the gate derivative
+        check_dz_codes("dZq", r.dZq, bw["dZq"], CODE_FRAC, OUT_TOL)
+    else:
+        frac, worst = code_mismatch(r.dZq, bw["dZq"])
+        assert worst <= 1 and frac <= CODE_FRAC, f"dZq codes: {frac:.2e} differ, worst {worst} steps"
     for name, got, ref in (("dX", bf16_bits_to_f32(r.dX_bits), bw["dX"]), ("dW1", r.dW1.cpu().numpy(), bw["dW1"]),
                            ("dW2", r.dW2.cpu().numpy(), bw["dW2"]), ("dW3", r.dW3.cpu().numpy(), bw["dW3"])):
         assert np.all(np.isfinite(got)), f"{name} has unwritten or non-finite entries"
@@ -135,6 +138,23 @@ def test_ragged_shapes_given_scales(shape):
             assert np.array_equal(r.scales[k], np.atleast_1d(np.asarray(v, np.float32)))
         check_forward(r, fw)
         check_backward(r, bw)
+    finally:
+        r.close()
+
+
+def test_ragged_shape_on_wide_tiles():
+    """The down projection and the input-gradient GEMM switch to 256 x 512 tiles once those fill the CTA pairs
+    (at least half as many tiles as SMs).  T = 2520 and d = 4048 give 10 x 8 such tiles with a ragged last row
+    of tiles (216 of 256 tokens) and a ragged last column of tiles (464 of 512 outputs); f stays small so that
+    the oracle finishes in seconds."""
+    T, d, f = 2520, 4048, 144
+    w = wl.make("wide", 21, T, d, f, w_std=0.05, channel_outlier_frac=0.01)
+    fw = oracle.forward(w.x, w.W1, w.W2, w.W3)
+    bw = oracle.backward(fw, w.dY)
+    r = Run(w, B.SMOOTH | B.SAVE_FOR_BWD, B.SCALE_FROM_CURRENT_AMAX)
+    try:
+        check_forward(r, fw)
+        check_backward(r, bw, many_codes=True)
     finally:
         r.close()
 
