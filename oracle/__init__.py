@@ -223,8 +223,10 @@ def forward(x_bf16, W1, W2, W3, *, flags: int = FLAG_SMOOTH, scale_mode: int = S
     return r
 
 
-def backward(fwd: dict, dy_bf16, *, scale_mode: int = SCALE_CURRENT, sdy=None, sdz=None) -> dict:
-    """Backward of the block from the dict forward() returned (same flags)."""
+def backward(fwd: dict, dy_bf16, *, scale_mode: int = SCALE_CURRENT, sdy=None, sdz=None,
+             want_intermediates: bool = False) -> dict:
+    """Backward of the block from the dict forward() returned (same flags).  want_intermediates adds the fp32
+    dH [T,f] and dZ = [dG | dU] [T,2f] as they stand before the E5M2 cast."""
     dy_bf16 = np.ascontiguousarray(dy_bf16, dtype=np.uint16)
     T, d, f, flags = fwd["T"], fwd["d"], fwd["f"], fwd["flags"]
     assert dy_bf16.shape == (T, d)
@@ -235,6 +237,8 @@ def backward(fwd: dict, dy_bf16, *, scale_mode: int = SCALE_CURRENT, sdy=None, s
     r = dict(dYq=np.empty((T, d), np.uint8), dZq=np.empty((T, 2 * f), np.uint8),
              dX_bits=np.empty((T, d), np.uint16), dX=np.empty((T, d), np.float32),
              dW1=np.empty((d, f), np.float32), dW2=np.empty((d, f), np.float32), dW3=np.empty((f, d), np.float32))
+    if want_intermediates:
+        r.update(dH=np.empty((T, f), np.float32), dZ=np.empty((T, 2 * f), np.float32))
     rc = lib().orc_backward(
         C.c_int64(T), C.c_int64(d), C.c_int64(f), C.c_uint(flags), C.c_int(scale_mode), _p(dy_bf16),
         _p(fwd["Xq"]), _p(fwd["W12q"]), _p(fwd["W3q"]), _p(fwd["Hq"]),
@@ -243,7 +247,7 @@ def backward(fwd: dict, dy_bf16, *, scale_mode: int = SCALE_CURRENT, sdy=None, s
         C.c_float(fwd["sx"]), C.c_float(fwd["sw12"]), _p(fwd["s_h"]), C.c_float(fwd["sw3"]),
         C.byref(c_sdy), C.byref(c_sdz), C.byref(a_dy), C.byref(a_dz),
         _p(r["dYq"]), _p(r["dZq"]), _p(r["dX_bits"]), _p(r["dX"]), _p(r["dW1"]), _p(r["dW2"]), _p(r["dW3"]),
-        _p(fwd.get("GUq")), C.c_float(fwd.get("sgu", 1.0)))
+        _p(fwd.get("GUq")), C.c_float(fwd.get("sgu", 1.0)), _p(r.get("dH")), _p(r.get("dZ")))
     assert rc == 0
     r.update(sdy=float(c_sdy.value), sdz=float(c_sdz.value), amax_dy=float(a_dy.value), amax_dz=float(a_dz.value))
     return r

@@ -159,8 +159,9 @@ void orc_f32_to_bf16_array(const float* v, int64_t n, uint16_t* out) {
 }
 
 /* ------------------------------------------------------------------ scaling (Section 2)
- * READING: "per-tensor scaling ... based on its specific range of values" is taken as
- * scale = fmt_max / max|v| with no margin; a zero or non-finite amax gives scale 1.
+ * READING: Section 2 describes per-tensor scaling only as a factor chosen from the range of the
+ * tensor's values; it is taken as scale = fmt_max / max|v| with no margin; a zero or non-finite
+ * amax gives scale 1.
  */
 float orc_amax(const float* v, int64_t n) {
     float a = 0.0f;
@@ -175,8 +176,8 @@ float orc_scale_from_amax(int fmt, float amax) {
     return s;
 }
 
-/* READING (Section 4.4, step 3 "use these per-channel maximum values to determine the
- * individual scaling factors"): s is the largest power of two p with p*amax <= fmt_max.
+/* READING (Section 4.4, third step of the recipe: the per-channel maxima decide the per-channel
+ * factors, no formula given): s is the largest power of two p with p*amax <= fmt_max.
  * A power of two makes s * s^-1 exact, so the scaled block is the same function.
  * fmt_max = 0.875 * 2^E with E = 9 (E4M3) or 16 (E5M2); amax = m * 2^e, m in [0.5, 1).
  */
@@ -386,8 +387,8 @@ int orc_forward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode,
     /* Q(s_i * H) (Eq. 2) */
     const int h_bf16 = (flags & ORC_FLAG_H_BF16) != 0;
     if (h_bf16) {
-        /* READING: "disabling the quantisation of the last linear layer" = that layer runs in bf16:
-         * H and W3 are rounded to bf16 (no scales), products accumulate in fp32. */
+        /* READING (Section 4.3: the experiment that leaves the last linear layer's input unquantised):
+         * that layer runs in bf16 - H and W3 are rounded to bf16 (no scales), products accumulate in fp32. */
         for (int64_t i = 0; i < f; ++i) s_h[i] = 1.0f;
         for (int64_t i = 0; i < T * f; ++i) {
             hq[i] = orc_bf16_to_f32(orc_f32_to_bf16(H[i]));
@@ -461,6 +462,8 @@ int orc_forward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode,
  * derived from max(|dG|,|dU|) in current-amax mode.
  * For ORC_FLAG_Q_IDENTITY the "codes" are unused and the decoded operands are passed as
  * fp32 arrays instead (xq_f, w12q_f [d,2f], w3q_f, hq_f).
+ * dH_out / dZ_out (nullable) receive the fp32 intermediates dH and [dG | dU] as they stand before
+ * the E5M2 cast (tests derive tolerance bounds from them; nothing else reads them).
  */
 int orc_backward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode,
                  const uint16_t* dy_bf16,
@@ -471,7 +474,8 @@ int orc_backward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode
                  float* sdy, float* sdz, float* amax_dy, float* amax_dz,
                  uint8_t* dYq, uint8_t* dZq /*[T,2f]: dG | dU*/,
                  uint16_t* dX_bf16, float* dX_f32, float* dW1, float* dW2, float* dW3,
-                 const uint8_t* GUq, float sgu) {
+                 const uint8_t* GUq, float sgu,
+                 float* dH_out /*[T,f], nullable*/, float* dZ_out /*[T,2f] = dG | dU before scaling, nullable*/) {
     const int smooth = (flags & ORC_FLAG_SMOOTH) != 0;
     const int qid = (flags & ORC_FLAG_Q_IDENTITY) != 0;
     float* dyf  = (float*)malloc(sizeof(float) * T * d);
@@ -543,6 +547,8 @@ int orc_backward(int64_t T, int64_t d, int64_t f, unsigned flags, int scale_mode
             orc_swiglu_grad(u, g, dh, &du, &dg);
             dG[t * f + i] = dg;
             dU[t * f + i] = du;
+            if (dH_out) dH_out[t * f + i] = dh;
+            if (dZ_out) { dZ_out[t * 2 * f + i] = dg; dZ_out[t * 2 * f + f + i] = du; }
             float a = fabsf(dg); if (a > adz) adz = a;
             a = fabsf(du);       if (a > adz) adz = a;
         }

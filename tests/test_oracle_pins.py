@@ -497,3 +497,36 @@ def test_gu_fp8_option_is_exact_when_the_activations_are_representable():
     bb = oracle.backward(b, dY, scale_mode=SCALE_GIVEN, sdy=64.0, sdz=8.0)
     for k in ("dZq", "dX_bits", "dW1", "dW2", "dW3"):
         assert np.array_equal(ba[k], bb[k]), k
+
+
+def test_backward_intermediates_are_what_the_codes_and_the_maximum_are_made_of():
+    """The optional fp32 outputs of the backward (dH and dZ = [dG | dU] before the E5M2 cast): a library cast of
+    sdz * dZ gives the stored codes, numpy's max |dZ| the reported maximum, and dZ follows from dH and the saved
+    activations by the element-wise gradient routine (pinned on its own against finite differences)."""
+    w = wl.make("im", 9, 24, 64, 96, w_std=0.05, channel_outlier_frac=0.02)
+    fw = oracle.forward(w.x, w.W1, w.W2, w.W3)
+    bw = oracle.backward(fw, w.dY, want_intermediates=True)
+    plain = oracle.backward(fw, w.dY)
+    assert np.array_equal(bw["dZq"], plain["dZq"]) and np.array_equal(bw["dW1"], plain["dW1"])   # asking changes nothing
+    assert np.float32(np.abs(bw["dZ"]).max()) == np.float32(bw["amax_dz"])
+    lib_codes = (torch.from_numpy(bw["dZ"] * np.float32(bw["sdz"])).to(torch.float8_e5m2)).view(torch.uint8).numpy()
+    assert np.array_equal(lib_codes, bw["dZq"])
+    g, u = oracle.bf16_to_f32(fw["G"]), oracle.bf16_to_f32(fw["U"])
+    f = w.f
+    for t, i in ((0, 0), (3, 17), (23, 95), (11, 40)):
+        du, dg = oracle.swiglu_grad(float(u[t, i]), float(g[t, i]), float(bw["dH"][t, i]))
+        assert np.float32(dg) == bw["dZ"][t, i] and np.float32(du) == bw["dZ"][t, f + i]
+
+
+def test_amax_dz_envelope_of_the_parity_tests():
+    """Host logic of the tolerance the GPU tests use for the maximum of dZ: with no storage step the envelope
+    collapses onto the oracle's maximum; with one bf16 step it contains it and stays within a few 2^-8."""
+    from helpers import amax_dz_bounds, bf16_ulp
+    w = wl.make("env", 10, 16, 64, 80, w_std=0.05)
+    fw = oracle.forward(w.x, w.W1, w.W2, w.W3)
+    bw = oracle.backward(fw, w.dY, want_intermediates=True)
+    g, u = oracle.bf16_to_f32(fw["G"]), oracle.bf16_to_f32(fw["U"])
+    lo, hi = amax_dz_bounds(g, u, bw["dH"], 0.0 * g, 0.0 * u)
+    assert lo == hi and np.isclose(lo, bw["amax_dz"], rtol=1e-6)
+    lo, hi = amax_dz_bounds(g, u, bw["dH"], bf16_ulp(g), bf16_ulp(u))
+    assert lo <= bw["amax_dz"] <= hi and hi / lo < 1.0 + 8 * 2.0 ** -7
