@@ -25,3 +25,23 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+# ---------------------------------------------------------------- parity report
+# Tests that compare the CUDA path with the oracle record the figures they measured (literal errors,
+# fractions of differing codes, how much each allowance was used) with record_parity(); the session
+# prints them and, if FP8MLP_PARITY_REPORT names a file, writes them there as JSON.
+from helpers import PARITY_FIGURES as _PARITY  # noqa: E402
+
+
+def pytest_terminal_summary(terminalreporter):
+    if not _PARITY:
+        return
+    import json
+    terminalreporter.write_sep("-", "parity figures")
+    for row in _PARITY:
+        terminalreporter.write_line(json.dumps(row))
+    path = os.environ.get("FP8MLP_PARITY_REPORT")
+    if path:
+        with open(path, "w") as fh:
+            json.dump(_PARITY, fh, indent=1)

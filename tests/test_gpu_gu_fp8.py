@@ -9,7 +9,8 @@ import pytest
 import torch
 
 import oracle
-from helpers import bf16_bits_to_f32, bf16_dev_to_bits, code_mismatch, nmax_err, nmax_err_bf16, to_dev, to_dev_bf16
+from helpers import (bf16_bits_to_f32, bf16_dev_to_bits, check_amax_dz, code_mismatch, e4m3_step, nmax_err, nmax_err_bf16,
+                     to_dev, to_dev_bf16)
 from paper_2409_12517_b200 import binding as B
 from paper_2409_12517_b200 import workloads as wl
 
@@ -57,7 +58,14 @@ def _check(r, fw, bw, given_scales):
     frac, worst = code_mismatch(r["Hq"], fw["Hq"])
     assert worst <= 1 and frac <= CODE_FRAC, f"Hq codes: {frac:.2e} differ, worst {worst} steps"
     assert nmax_err_bf16(r["Y"], fw["Y"]) <= OUT_TOL, "Y"
-    assert np.isclose(r["am"]["dz"][0], bw["amax_dz"], rtol=1e-3), "amax of dZ"
+    # the saved activations are E4M3 codes here: where a stored code differs from the oracle's (by one step: checked
+    # above) the maximum of dZ is held to the envelope that step opens, elsewhere to the accumulation-order bar
+    gu = oracle.decode(oracle.E4M3, fw["GUq"]).astype(np.float64)
+    f = gu.shape[1] // 2
+    inv = 1.0 / float(fw["sgu"])
+    differs = r["GUq"] != fw["GUq"]                      # the step is granted only where the stored code differs
+    check_amax_dz("amax of dZ", r["am"]["dz"][0], bw, gu[:, :f] * inv, gu[:, f:] * inv,
+                  np.where(differs[:, :f], e4m3_step(gu[:, :f]), 0.0) * inv, np.where(differs[:, f:], e4m3_step(gu[:, f:]), 0.0) * inv)
     assert r["sc"]["dz"][0] == np.float32(bw["sdz"]), "scale of dZ"
     frac, worst = code_mismatch(r["dZq"], bw["dZq"])
     assert worst <= 1 and frac <= CODE_FRAC, f"dZq codes: {frac:.2e} differ, worst {worst} steps"
@@ -74,7 +82,7 @@ def test_gu_fp8_current_amax(cfg, smooth):
     w = wl.make_config("tiny") if cfg == "tiny" else wl.make("gu8", 41, *cfg, w_std=0.05, channel_outlier_frac=0.01)
     ofl = (oracle.FLAG_SMOOTH if smooth else 0) | oracle.FLAG_GU_FP8
     fw = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=ofl)
-    bw = oracle.backward(fw, w.dY)
+    bw = oracle.backward(fw, w.dY, want_intermediates=True)
     r = _run(w, B.SMOOTH if smooth else 0, B.SCALE_FROM_CURRENT_AMAX)
     _check(r, fw, bw, given_scales=False)
 
@@ -92,7 +100,7 @@ def test_gu_fp8_given_scales(shape):
     given = dict(x=pf["sx"], w12=pf["sw12"], w3=pf["sw3"], h=pf["s_h"], dy=pb["sdy"], dz=pb["sdz"], gu=pf["sgu"])
     fw = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=ofl, scale_mode=oracle.SCALE_GIVEN, sx=pf["sx"],
                         sw12=pf["sw12"], s_h=pf["s_h"], sw3=pf["sw3"], sgu=pf["sgu"])
-    bw = oracle.backward(fw, w.dY, scale_mode=oracle.SCALE_GIVEN, sdy=pb["sdy"], sdz=pb["sdz"])
+    bw = oracle.backward(fw, w.dY, scale_mode=oracle.SCALE_GIVEN, sdy=pb["sdy"], sdz=pb["sdz"], want_intermediates=True)
     r = _run(w, B.SMOOTH, B.SCALE_GIVEN, given=given)
     _check(r, fw, bw, given_scales=True)
 

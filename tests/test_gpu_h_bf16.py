@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import (bf16_bits_to_f32, bf16_dev_to_bits, code_mismatch, nmax_err, nmax_err_bf16, to_dev, to_dev_bf16)
+from helpers import (bf16_bits_to_f32, bf16_dev_to_bits, bf16_ulp, check_amax_dz, code_mismatch, nmax_err, nmax_err_bf16, to_dev, to_dev_bf16)
 from paper_2409_12517_b200 import binding as B
 from paper_2409_12517_b200 import workloads as wl
 
@@ -37,7 +37,7 @@ def test_h_bf16_forward_backward(cfg, mode):
     w = wl.make_config("tiny") if cfg == "tiny" else wl.make("hb", 31, *cfg, w_std=0.05, channel_outlier_frac=0.01)
     T, d, f = w.T, w.d, w.f
     fw = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=oracle.FLAG_H_BF16, want_float_operands=True)
-    bw = oracle.backward(fw, w.dY)
+    bw = oracle.backward(fw, w.dY, want_intermediates=True)
     ctx = B.fp8mlp_create(T, d, f, B.H_BF16 | B.SAVE_FOR_BWD)
     try:
         sc, am = B.new_scales(f), B.new_amax(f)
@@ -58,7 +58,11 @@ def test_h_bf16_forward_backward(cfg, mode):
         hb = ws(B.WS_HB, (T, f), torch.int16).view(np.uint16)
         assert nmax_err_bf16(hb, fw["hq_f"]) <= 1e-5, "H in bf16"
         assert nmax_err_bf16(bf16_dev_to_bits(y), fw["Y"]) <= 2e-3, "Y"
-        assert np.isclose(am["dz"].item(), bw["amax_dz"], rtol=1e-3) and sc["dz"].item() == np.float32(bw["sdz"])
+        g, u = bf16_bits_to_f32(fw["G"]), bf16_bits_to_f32(fw["U"])
+        gu = ws(B.WS_GU, (T, 2 * f), torch.int16).view(np.uint16)
+        check_amax_dz("amax of dZ", am["dz"].item(), bw, g, u, np.where(gu[:, :f] != fw["G"], bf16_ulp(g), 0.0),
+                      np.where(gu[:, f:] != fw["U"], bf16_ulp(u), 0.0))      # one spacing where the saved value differs
+        assert sc["dz"].item() == np.float32(bw["sdz"])
         frac, worst = code_mismatch(ws(B.WS_DZQ, (T, 2 * f)), bw["dZq"])
         assert worst <= 1 and frac <= 1e-3, f"dZq codes: {frac:.2e} differ, worst {worst}"
         assert nmax_err_bf16(bf16_dev_to_bits(dx), bw["dX"]) <= 2e-3, "dX"

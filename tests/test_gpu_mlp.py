@@ -9,7 +9,8 @@ import pytest
 import torch
 
 import oracle
-from helpers import bf16_dev_to_bits, bf16_bits_to_f32, check_dz_codes, code_mismatch, nmax_err, to_dev, to_dev_bf16
+from helpers import (bf16_dev_to_bits, bf16_bits_to_f32, bf16_ulp, check_amax_dz, check_dz_codes, code_mismatch, nmax_err,
+                     nmax_err_bf16, record_parity, to_dev, to_dev_bf16)
 from paper_2409_12517_b200 import binding as B
 from paper_2409_12517_b200 import workloads as wl
 
@@ -76,17 +77,26 @@ def check_forward(r: Run, fw: dict, save=True):
     frac, worst = code_mismatch(r.Hq, fw["Hq"])
     assert worst <= 1 and frac <= CODE_FRAC, f"Hq codes: {frac:.2e} differ, worst {worst} steps"
     if save:
+        # element by element: the two fp32 values differ in accumulation order only, so their bf16 roundings are
+        # equal or, across a rounding boundary, one spacing apart
         for name, got, ref in (("G", r.GU[:, :f], fw["G"]), ("U", r.GU[:, f:], fw["U"])):
-            e = nmax_err(bf16_bits_to_f32(got), bf16_bits_to_f32(ref))
-            assert e <= 2.0 ** -8, f"saved {name}: {e}"
+            e = nmax_err_bf16(got, bf16_bits_to_f32(ref))
+            assert e <= 1e-5, f"saved {name}: {e} beyond one bf16 spacing"
     e = nmax_err(bf16_bits_to_f32(r.Y_bits), fw["Y"])
     assert e <= OUT_TOL, f"Y: {e}"
 
 
-def check_backward(r: Run, bw: dict, many_codes: bool = False):
+def check_backward(r: Run, fw: dict, bw: dict, many_codes: bool = False):
     assert r.amax["dy"][0] == np.float32(bw["amax_dy"]) and r.scales["dy"][0] == np.float32(bw["sdy"])
     assert np.array_equal(r.dYq, bw["dYq"]), "dY codes differ"
-    assert np.isclose(r.amax["dz"][0], bw["amax_dz"], rtol=1e-3), "amax of dZ"
+    # the accumulation-order bar, opened by one bf16 spacing only at the elements whose saved G or U does differ
+    # from the oracle's (those have passed their own bar: at most one spacing)
+    f = r.w.f
+    g, u = bf16_bits_to_f32(fw["G"]), bf16_bits_to_f32(fw["U"])
+    g_step = np.where(r.GU[:, :f] != fw["G"], bf16_ulp(g), 0.0)
+    u_step = np.where(r.GU[:, f:] != fw["U"], bf16_ulp(u), 0.0)
+    record_parity("amax_dz " + r.w.name, saved_activations_differing=int(np.count_nonzero(g_step) + np.count_nonzero(u_step)),
+                  **check_amax_dz("amax of dZ", r.amax["dz"][0], bw, g, u, g_step, u_step, AMAX_RTOL))
     assert r.scales["dz"][0] == np.float32(bw["sdz"]), "scale of dZ"
     if many_codes:      # among hundreds of thousands of codes a few sit at the zero of the gate derivative
         check_dz_codes("dZq", r.dZq, bw["dZq"], CODE_FRAC, OUT_TOL)
@@ -110,11 +120,11 @@ def test_tiny_config_current_amax(flags):
     current amax, Smooth-SwiGLU on and off."""
     w = wl.make_config("tiny")
     fw = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=_oracle_flags(flags))
-    bw = oracle.backward(fw, w.dY)
+    bw = oracle.backward(fw, w.dY, want_intermediates=True)
     r = Run(w, flags, B.SCALE_FROM_CURRENT_AMAX)
     try:
         check_forward(r, fw)
-        check_backward(r, bw)
+        check_backward(r, fw, bw)
     finally:
         r.close()
 
@@ -131,13 +141,13 @@ def test_ragged_shapes_given_scales(shape):
     given = dict(x=pf["sx"], w12=pf["sw12"], w3=pf["sw3"], h=pf["s_h"], dy=pb["sdy"], dz=pb["sdz"])
     fw = oracle.forward(w.x, w.W1, w.W2, w.W3, scale_mode=oracle.SCALE_GIVEN, sx=pf["sx"], sw12=pf["sw12"],
                         s_h=pf["s_h"], sw3=pf["sw3"])
-    bw = oracle.backward(fw, w.dY, scale_mode=oracle.SCALE_GIVEN, sdy=pb["sdy"], sdz=pb["sdz"])
+    bw = oracle.backward(fw, w.dY, scale_mode=oracle.SCALE_GIVEN, sdy=pb["sdy"], sdz=pb["sdz"], want_intermediates=True)
     r = Run(w, B.SMOOTH | B.SAVE_FOR_BWD, B.SCALE_GIVEN, given=given)
     try:
         for k, v in given.items():                       # given scales are left alone
             assert np.array_equal(r.scales[k], np.atleast_1d(np.asarray(v, np.float32)))
         check_forward(r, fw)
-        check_backward(r, bw)
+        check_backward(r, fw, bw)
     finally:
         r.close()
 
@@ -150,11 +160,11 @@ def test_ragged_shape_on_wide_tiles():
     T, d, f = 2520, 4048, 144
     w = wl.make("wide", 21, T, d, f, w_std=0.05, channel_outlier_frac=0.01)
     fw = oracle.forward(w.x, w.W1, w.W2, w.W3)
-    bw = oracle.backward(fw, w.dY)
+    bw = oracle.backward(fw, w.dY, want_intermediates=True)
     r = Run(w, B.SMOOTH | B.SAVE_FOR_BWD, B.SCALE_FROM_CURRENT_AMAX)
     try:
         check_forward(r, fw)
-        check_backward(r, bw, many_codes=True)
+        check_backward(r, fw, bw, many_codes=True)
     finally:
         r.close()
 

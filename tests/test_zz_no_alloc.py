@@ -2,20 +2,22 @@
 
 Such callers (a plug-in inside an application whose pool owns the whole GPU, a serving loop that
 must avoid the stalls of cudaMalloc / cudaFree) have no context; the library's fixed 4 MiB scratch
-array takes its place.  This checks, through the C ABI, that the entry point gives what
-fp8mlp_forward gives, on two calls in a row (the array keeps the first call's leftovers), and that
-shapes beyond the array are refused before anything runs.  Collected last on purpose.
+array takes its place.  This checks, through the C ABI, that the entry point gives exactly what
+fp8mlp_forward gives (bit for bit, and within the oracle's bar), on calls in a row (the array keeps the previous
+call's leftovers), that a call leaves the amount of free device memory unchanged, and that shapes beyond the
+array and bad arguments are refused before anything runs.  Collected last on purpose.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from helpers import bf16_bits_to_f32, bf16_dev_to_bits, nmax_err, to_dev, to_dev_bf16
 from paper_2409_12517_b200 import binding as B
 from paper_2409_12517_b200 import build as libbuild
 from paper_2409_12517_b200 import workloads as wl
 
-OUT_TOL = 2e-3      # the bar the other parity tests use for outputs
+OUT_TOL = 2e-3      # the bar the other parity tests use for outputs against the oracle
 
 
 def _forward_with_context(w, flags, mode, sc, am):
@@ -31,10 +33,12 @@ def _forward_with_context(w, flags, mode, sc, am):
 
 @pytest.mark.gpu
 def test_static_forward_matches_the_context_forward_twice_in_a_row():
-    # two different problems back to back: the second finds the first one's data in the scratch
+    """Same kernels on the same data: the result must equal fp8mlp_forward's bit for bit (outputs, scales and
+    maxima), in both scale modes, and the first problem's result must also meet the oracle's bar."""
+    # different problems back to back: each finds the previous one's data in the scratch
     problems = [(wl.make_config("tiny"), B.SMOOTH), (wl.make("second", 5, 200, 128, 400, w_std=0.05), B.SMOOTH),
                 (wl.make_config("tiny"), 0)]
-    for w, flags in problems:
+    for n, (w, flags) in enumerate(problems):
         sc_ref, am_ref = B.new_scales(w.f), B.new_amax(w.f)
         y_ref = _forward_with_context(w, flags, B.SCALE_FROM_CURRENT_AMAX, sc_ref, am_ref)
         for mode in (B.SCALE_FROM_CURRENT_AMAX, B.SCALE_GIVEN):
@@ -46,13 +50,42 @@ def test_static_forward_matches_the_context_forward_twice_in_a_row():
             B.fp8mlp_forward_static(w.T, w.d, w.f, flags, to_dev_bf16(w.x), to_dev(w.W1), to_dev(w.W2), to_dev(w.W3),
                                     mode, sc, am, y)
             torch.cuda.synchronize()
-            got = bf16_bits_to_f32(bf16_dev_to_bits(y))
-            assert np.all(np.isfinite(got))
-            assert nmax_err(got, bf16_bits_to_f32(y_ref)) <= OUT_TOL
+            got_bits = bf16_dev_to_bits(y)
+            assert np.array_equal(got_bits, y_ref), "output differs from fp8mlp_forward's"
             for k in ("x", "w12", "w3", "h"):
-                assert torch.allclose(sc[k], sc_ref[k], rtol=1e-5, atol=0)
+                assert torch.equal(sc[k], sc_ref[k]), f"scale {k}"
             for k in ("x", "w1", "w2", "w3", "h"):
-                assert torch.allclose(am[k], am_ref[k], rtol=1e-5, atol=0)
+                assert torch.equal(am[k], am_ref[k]), f"maximum {k}"
+            if n == 0 and mode == B.SCALE_FROM_CURRENT_AMAX:      # and against the CPU oracle, once
+                fw = oracle.forward(w.x, w.W1, w.W2, w.W3, flags=oracle.FLAG_SMOOTH)
+                assert np.array_equal(sc["h"].cpu().numpy(), fw["s_h"])
+                assert nmax_err(bf16_bits_to_f32(got_bits), fw["Y"]) <= OUT_TOL
+
+
+@pytest.mark.gpu
+def test_static_forward_leaves_device_memory_as_it_found_it():
+    """The promise to callers that cannot allocate: once the library is loaded and the kernels have run once,
+    a call takes no device memory - the free bytes the driver reports are the same before and after."""
+    w = wl.make_config("tiny")
+    x, W1, W2, W3 = to_dev_bf16(w.x), to_dev(w.W1), to_dev(w.W2), to_dev(w.W3)
+    sc, am = B.new_scales(w.f), B.new_amax(w.f)
+    y = torch.zeros((w.T, w.d), dtype=torch.bfloat16, device="cuda")
+    call = lambda: B.fp8mlp_forward_static(w.T, w.d, w.f, B.SMOOTH, x, W1, W2, W3, B.SCALE_FROM_CURRENT_AMAX, sc, am, y)
+    call()                                   # warm-up: the runtime loads the kernels and sets the array up
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    call()
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, f"device memory in use changed by {free_before - free_after} bytes across the call"
+    # a bad argument (here: x not 16-byte aligned, then no scales) is refused before anything is enqueued
+    n0 = B.fp8mlp_launch_count()
+    with pytest.raises(B.Fp8MlpError) as ei:
+        B.fp8mlp_forward_static(w.T, w.d, w.f, B.SMOOTH, x.view(-1)[4:4 + w.T * w.d], W1, W2, W3, B.SCALE_GIVEN, sc, am, y)
+    assert ei.value.code == B.ERR_ALIGN
+    assert B.lib().fp8mlp_forward_static(w.T, w.d, w.f, B.SMOOTH, x.data_ptr(), W1.data_ptr(), W2.data_ptr(), W3.data_ptr(),
+                                         B.SCALE_GIVEN, None, None, y.data_ptr(), None) == B.ERR_ARG
+    assert B.fp8mlp_launch_count() == n0
 
 
 def test_static_forward_rejects_what_does_not_fit():
