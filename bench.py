@@ -69,56 +69,111 @@ def load_peaks():
 
 # ---------------------------------------------------------------- clocks sampler
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """SM clock, power and clock-event reasons of one GPU while the benchmark runs, read through NVML from a
+    thread of this process every 10 ms (only reads: no setting is touched).  The record spans the warm-up and
+    the timed region; summary() reports the timed region and the whole window separately.  Falls back to
+    polling nvidia-smi when the NVML binding is missing."""
 
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    PERIOD_S = 0.010
+    SMI_FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+                  "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+                  "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.rows, self.proc, self.thread, self.gpu = [], None, None, gpu_index
+    def __init__(self, gpu_index: int, uuid: str | None = None):
+        self.rows = []                    # (time, sm_mhz, watts, set of reason names)
+        self.gpu, self.uuid = gpu_index, uuid
+        self.max_mhz, self.how = None, None
+        self._stop = threading.Event()
+        self.thread, self.proc = None, None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+            import pynvml as N
+            N.nvmlInit()
+            h = None
+            if self.uuid:
+                try:
+                    h = N.nvmlDeviceGetHandleByUUID(self.uuid if self.uuid.startswith("GPU-") else "GPU-" + self.uuid)
+                except N.NVMLError:
+                    h = None
+            if h is None:
+                h = N.nvmlDeviceGetHandleByIndex(self.gpu)
+            self.max_mhz = float(N.nvmlDeviceGetMaxClockInfo(h, N.NVML_CLOCK_SM))
+            names = (("hw_slowdown", N.nvmlClocksEventReasonHwSlowdown), ("hw_thermal_slowdown", N.nvmlClocksEventReasonHwThermalSlowdown),
+                     ("sw_thermal_slowdown", N.nvmlClocksEventReasonSwThermalSlowdown), ("sw_power_cap", N.nvmlClocksEventReasonSwPowerCap),
+                     ("hw_power_brake", N.nvmlClocksEventReasonHwPowerBrakeSlowdown))
+
+            def poll():
+                while not self._stop.is_set():
+                    try:
+                        mhz = float(N.nvmlDeviceGetClockInfo(h, N.NVML_CLOCK_SM))
+                        watts = N.nvmlDeviceGetPowerUsage(h) / 1000.0
+                        mask = N.nvmlDeviceGetCurrentClocksEventReasons(h)
+                        self.rows.append((time.time(), mhz, watts, {n for n, bit in names if mask & bit}))
+                    except N.NVMLError:
+                        pass
+                    self._stop.wait(self.PERIOD_S)
+
+            self.how = f"NVML, one read per {int(self.PERIOD_S * 1e3)} ms"
+            self.thread = threading.Thread(target=poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            pass
+        try:                              # fallback: nvidia-smi as fast as it will go
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.SMI_FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
-        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.how = "nvidia-smi -lms 100"
+
+        def read():
+            num = lambda v: float(v) if v.replace(".", "", 1).isdigit() else None
+            for line in self.proc.stdout:
+                c = [x.strip() for x in line.split(",")]
+                if len(c) < 7 or num(c[0]) is None:
+                    continue
+                self.max_mhz = num(c[1])
+                reasons = {n for n, col in (("hw_slowdown", 3), ("hw_thermal_slowdown", 4), ("sw_thermal_slowdown", 5),
+                                            ("sw_power_cap", 6)) if c[col].lower().startswith("active")}
+                self.rows.append((time.time(), num(c[0]), num(c[2]), reasons))
+
+        self.thread = threading.Thread(target=read, daemon=True)
         self.thread.start()
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+    def stop(self):
+        self._stop.set()
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
 
-    def stop(self, t0: float, t1: float) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        good = [(t, r) for t, r in self.rows if len(r) >= 8]
-        rows = [r for t, r in good if t0 <= t <= t1]
-        if not rows and good:            # a timed region shorter than the sampling period: the sample nearest to it
-            rows = [min(good, key=lambda tr: min(abs(tr[0] - t0), abs(tr[0] - t1)))[1]]
+    def window(self, t0: float, t1: float) -> dict:
+        rows = [r for r in self.rows if t0 <= r[0] <= t1]
         if not rows:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        num = lambda s: float(s) if s.replace(".", "", 1).isdigit() else None
-        sm = sorted(v for v in (num(r[0]) for r in rows) if v is not None)
-        reasons = set()
-        for r in rows:
-            for name, col in (("hw_slowdown", 4), ("hw_thermal_slowdown", 5), ("sw_thermal_slowdown", 6), ("sw_power_cap", 7)):
-                if r[col].lower().startswith("active"):
-                    reasons.add(name)
-        power = [v for v in (num(r[2]) for r in rows) if v is not None]
-        masks = sorted({r[3] for r in rows})
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": num(rows[0][1]), "active_masks": masks,
-                "power_w_max": max(power) if power else None, "samples": len(rows), "reasons": sorted(reasons)}
+            return {"samples": 0}
+        mhz = sorted(r[1] for r in rows)
+        watts = [r[2] for r in rows if r[2] is not None]
+        reasons = sorted(set().union(*[r[3] for r in rows]))
+        return {"samples": len(rows), "sm_mhz": mhz[len(mhz) // 2], "sm_mhz_min": mhz[0], "sm_mhz_max": mhz[-1],
+                "power_w_max": max(watts) if watts else None, "reasons": reasons,
+                "sw_power_cap_samples": sum(1 for r in rows if "sw_power_cap" in r[3])}
+
+    def summary(self, t_warm: float, t0: float, t1: float) -> dict:
+        """The contract's keys describe the timed region [t0, t1]; `warmup_and_timed` the window from the first
+        warm-up step to the end of the timed region."""
+        if self.how is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source (NVML binding and nvidia-smi both unavailable)"]}
+        timed, whole = self.window(t0, t1), self.window(t_warm, t1)
+        return {"sm_mhz": timed.get("sm_mhz"), "sm_max_mhz": self.max_mhz, "reasons": timed.get("reasons", []),
+                "samples": timed["samples"], "power_w_max": timed.get("power_w_max"), "timed_region": timed,
+                "warmup_and_timed": whole, "source": self.how}
 
 
 # ---------------------------------------------------------------- CPU oracle timing
@@ -177,6 +232,136 @@ def run_reference(args, rank: int):
     }))
 
 
+# ---------------------------------------------------------------- vendor FP8 GEMM (yardstick only)
+def vendor_fp8_gemm_rates(T: int, d: int, f: int, seconds: float = 2.0):
+    """What the vendor's FP8 GEMM (cuBLASLt through torch._scaled_mm) reaches on this GPU at the six (M, N, K) of the
+    step: a measured tensor-core ceiling to set beside the kernels of this repository.  Never part of the hot
+    path or of `value`.  E4M3 x E4M3 operands with K contiguous (the only layout that routine takes), per-tensor
+    scales, bf16 output (fp32 for the weight-gradient shapes).  Sustained: the six GEMMs back to back for
+    `seconds`, like the step itself, rates over the second half; after idle: best single call after 1 s of rest."""
+    import torch
+    shapes = {"gemm1_swiglu": (T, 2 * f, d), "gemm2_down": (T, d, f), "dgrad2_swiglu_bwd": (T, f, d),
+              "wgrad3": (f, d, T), "dgrad1": (T, d, 2 * f), "wgrad12": (d, 2 * f, T)}
+    one = torch.ones((), device="cuda")
+    ops = {}
+    try:
+        for name, (M, N, K) in shapes.items():
+            a = (torch.randn(M, K, device="cuda", dtype=torch.bfloat16) * 0.5).to(torch.float8_e4m3fn)
+            b = (torch.randn(N, K, device="cuda", dtype=torch.bfloat16) * 0.5).to(torch.float8_e4m3fn)
+            out_dtype = torch.float32 if name.startswith("wgrad") else torch.bfloat16
+            ops[name] = (a, b.t(), out_dtype, 2.0 * M * N * K)
+            torch._scaled_mm(a, b.t(), scale_a=one, scale_b=one, out_dtype=out_dtype)
+        torch.cuda.synchronize()
+    except Exception as exc:          # a build of torch without this routine, or a layout it refuses
+        return {"unavailable": f"{type(exc).__name__}: {exc}"[:200]}
+    run = lambda n: torch._scaled_mm(ops[n][0], ops[n][1], scale_a=one, scale_b=one, out_dtype=ops[n][2])
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    after_idle = {}
+    for name in ops:
+        best = float("inf")
+        for _ in range(2):
+            torch.cuda.synchronize()
+            time.sleep(1.0)
+            e0, e1 = ev(), ev()
+            e0.record(); run(name); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        after_idle[name] = round(ops[name][3] / (best * 1e-3) / 1e12, 1)
+    rounds, t_end = [], time.time() + seconds
+    while time.time() < t_end:
+        marks = [ev() for _ in range(len(ops) + 1)]
+        marks[0].record()
+        for i, name in enumerate(ops):
+            run(name)
+            marks[i + 1].record()
+        rounds.append(marks)
+        if len(rounds) % 8 == 0:
+            torch.cuda.synchronize()          # keeps the queue short so that the wall clock bounds the loop
+    torch.cuda.synchronize()
+    late = rounds[len(rounds) // 2:]
+    sustained, tot_ms, tot_flop = {}, 0.0, 0.0
+    for i, name in enumerate(ops):
+        ms = sum(m[i].elapsed_time(m[i + 1]) for m in late) / len(late)
+        sustained[name] = round(ops[name][3] / (ms * 1e-3) / 1e12, 1)
+        tot_ms += ms
+        tot_flop += ops[name][3]
+    return {"what": "torch._scaled_mm (cuBLASLt), E4M3 x E4M3, K-contiguous operands, at the six (M, N, K) of the step",
+            "sustained_tflops": sustained, "after_idle_tflops": after_idle, "rounds": len(rounds),
+            "sustained_all_six_tflops": round(tot_flop / (tot_ms * 1e-3) / 1e12, 1)}
+
+
+# ---------------------------------------------------------------- forward-only workloads
+def run_forward_only(args, rank: int, local_rank: int):
+    """Workloads without an output gradient (the 7B forward-only configuration, T = 4096): the forward of the block
+    with Smooth-SwiGLU on and off, delayed scaling (timed like the training step) and just-in-time scaling, and
+    what the per-channel scaling does to the SwiGLU codes: how many flush to zero, how many sit at the format's
+    largest value.  TFLOP/s = 6*T*d*f / time.  Output quality against the unquantised block is a test's job
+    (tests/test_gpu_full_size.py), not the benchmark's."""
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+
+    from paper_2409_12517_b200 import binding as B
+    from paper_2409_12517_b200 import build as libbuild
+    from paper_2409_12517_b200 import workloads as wl
+
+    torch.cuda.set_device(local_rank)
+    libbuild.build()
+    w = wl.make_config(args.workload)
+    T, d, f = w.T, w.d, w.f
+    x = torch.from_numpy(w.x.view(np.int16)).cuda().view(torch.bfloat16)
+    W1, W2, W3 = (torch.from_numpy(a).cuda() for a in (w.W1, w.W2, w.W3))
+    y = torch.empty_like(x)
+    flops = 6.0 * T * d * f
+    rows = {}
+    for smooth in (True, False):
+        ctx = B.fp8mlp_create(T, d, f, B.SMOOTH if smooth else 0)
+        sc, am = B.new_scales(f), B.new_amax(f)
+
+        def fwd(mode):
+            B.fp8mlp_forward(ctx, T, x, W1, W2, W3, mode, sc, am, y)
+            if mode == B.SCALE_GIVEN:
+                B.fp8mlp_update_scales(ctx, am, sc)
+
+        def timed(mode, n):
+            for _ in range(max(3, args.warmup)):
+                fwd(mode)
+            marks = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+            torch.cuda.synchronize()
+            marks[0].record()
+            for i in range(n):
+                fwd(mode)
+                marks[i + 1].record()
+            torch.cuda.synchronize()
+            per = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(n))
+            return marks[0].elapsed_time(marks[-1]) / n, per[n // 2]
+
+        fwd(B.SCALE_FROM_CURRENT_AMAX)
+        n0 = B.fp8mlp_launch_count()
+        mean_ms, med_ms = timed(B.SCALE_GIVEN, args.steps)
+        launches = B.fp8mlp_launch_count() - n0
+        jit_mean, jit_med = timed(B.SCALE_FROM_CURRENT_AMAX, min(args.steps, 50))
+        fwd(B.SCALE_FROM_CURRENT_AMAX)
+        assert B.fp8mlp_status(ctx) == B.OK
+        mag = B.workspace_tensor(ctx, B.WS_HQ, (T, f), torch.uint8) & 0x7F
+        rows["smooth_on" if smooth else "smooth_off"] = {
+            "ms": round(mean_ms, 4), "ms_median": round(med_ms, 4), "tflops": round(flops / (mean_ms * 1e-3) / 1e12, 1),
+            "just_in_time_ms": round(jit_mean, 4), "just_in_time_tflops_useful": round(flops / (jit_mean * 1e-3) / 1e12, 1),
+            "zero_code_frac": float((mag == 0).float().mean()), "largest_code_frac": float((mag == 0x7E).float().mean()),
+            "channels_whose_top_code_is_in_the_top_binade": int((mag.max(dim=0).values >= 0x76).sum()),
+            "gpu_launches": launches}
+        B.fp8mlp_destroy(ctx)
+    on = rows["smooth_on"]
+    print(json.dumps({
+        "metric": "FP8 Smooth-SwiGLU MLP forward TFLOP/s (6*T*d*f / time)", "value": on["tflops"], "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": on["ms"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "fp8 (E4M3, fp32 accumulate)", "data": "synthetic",
+        "config": {"workload": args.workload, "T": T, "d_model": d, "d_ff": f, "forward_only": True,
+                   "l2": "inputs per step (fp32 master weights 541 MB at the 7B shape) exceed the 126 MB L2"},
+        "gpu_launches": on["gpu_launches"], "rows": rows}))
+
+
 # ---------------------------------------------------------------- the CUDA arm
 def run_ours(args, rank: int, world: int, local_rank: int):
     import numpy as np
@@ -208,6 +393,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     def step(mode=B.SCALE_GIVEN):
         B.fp8mlp_forward(ctx, T, x, W1, W2, W3, mode, sc, am, y)
         B.fp8mlp_backward(ctx, T, dy, mode, sc, am, dx, dW1, dW2, dW3)
+        if mode == B.SCALE_GIVEN:
+            # delayed scaling's bookkeeping: this step's maxima become the next step's scales
+            B.fp8mlp_update_scales(ctx, am, sc)
 
     def barrier():
         torch.cuda.synchronize()
@@ -217,34 +405,41 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     # the "previous iteration" that delayed scaling takes its scales from: one just-in-time step
     step(B.SCALE_FROM_CURRENT_AMAX)
+    sampler = ClockSampler(local_rank, str(getattr(torch.cuda.get_device_properties(local_rank), "uuid", "")) or None)
+    if rank == 0:
+        sampler.start()
+    torch.cuda.synchronize()
+    t_warm = time.time()
     for _ in range(args.warmup):
         step()
     assert B.fp8mlp_status(ctx) == B.OK
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.25)
     B.fp8mlp_profile_enable(ctx, True)
     B.fp8mlp_profile_read(ctx)
     barrier()
     n0 = B.fp8mlp_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    e0, e1 = marks[0], marks[-1]
     t_wall0 = time.time()
-    e0.record()
-    for _ in range(args.steps):
+    marks[0].record()
+    for i in range(args.steps):
         step()
-    e1.record()
+        marks[i + 1].record()
     barrier()
     t_wall1 = time.time()
     launches = B.fp8mlp_launch_count() - n0
     ms_total = e0.elapsed_time(e1)
+    per_step = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
+    ms_median = per_step[len(per_step) // 2]
     prof = B.fp8mlp_profile_read(ctx)
     B.fp8mlp_profile_enable(ctx, False)
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    if rank == 0:
+        sampler.stop()
+    clocks = sampler.summary(t_warm, t_wall0, t_wall1) if rank == 0 else None
     assert B.fp8mlp_status(ctx) == B.OK
     ms_step = max_over_ranks(ms_total, world, "cuda") / args.steps
     value = job_tflops(T, d, f, world, ms_step)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     # The same kernels with a fresh power budget: single steps, each after a second of idle, so the board has not
     # yet throttled.  Context for the sustained figures above (which are what the metric is): not part of value.
@@ -306,6 +501,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                 main.wait_event(ev_out[b])                   # step i-2's results have left this output buffer
             B.fp8mlp_forward(ctx, T, xb[b], W1, W2, W3, B.SCALE_GIVEN, sc, am, yb[b])
             B.fp8mlp_backward(ctx, T, dyb[b], B.SCALE_GIVEN, sc, am, dxb[b], dW1, dW2, dW3)
+            B.fp8mlp_update_scales(ctx, am, sc)
             ev_comp[b].record(main)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_comp[b])
@@ -414,6 +610,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         B.fp8mlp_destroy(ctx0)
     if rank != 0:
         return
+    del dW1, dW2, dW3, W1, W2, W3
+    torch.cuda.empty_cache()
+    vendor = None if args.no_vendor_gemm else vendor_fp8_gemm_rates(T, d, f)
 
     peaks, peak_kind = load_peaks()
     fp8_peak = FP8_OVER_BF16 * peaks["bf16_tflops_sustained"]       # kernels timed inside a long step
@@ -424,6 +623,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     # with given scales the three weight matrices are quantised by one launch, reported as quant_w12
     phase_bytes = {"quant_x": 3.0 * T * d, "quant_dy": 3.0 * T * d, "quant_w12": 5.0 * 3 * d * f}
     kernels = {}
+    vendor_sus = (vendor or {}).get("sustained_tflops", {})
+    mhz = (clocks or {}).get("sm_mhz")
+    mhz_max = (clocks or {}).get("sm_max_mhz")
     for name, (ms, cnt) in prof.items():
         if cnt == 0:
             continue
@@ -432,17 +634,35 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         if name in phase_flops:
             entry["tflops"] = round(phase_flops[name] / (avg * 1e-3) / 1e12, 1)
             entry["frac_of_fp8_peak"] = round(entry["tflops"] / fp8_peak, 3)
+            entry["frac_of_nominal_fp8_4500"] = round(entry["tflops"] / NOMINAL_FP8_TFLOPS, 3)
+            if name in vendor_sus:
+                entry["frac_of_measured_fp8"] = round(entry["tflops"] / vendor_sus[name], 3)
+            if mhz and mhz_max:      # the same cycle count at the clock the board would hold without its power cap
+                entry["tflops_if_clock_held_at_max"] = round(entry["tflops"] * mhz_max / mhz, 1)
         if name in phase_bytes:
             entry["gbs"] = round(phase_bytes[name] / (avg * 1e-3) / 1e9, 1)
             entry["frac_of_hbm_peak"] = round(entry["gbs"] / peaks["hbm_gbs"], 3)
+            entry["frac_of_nominal_hbm_8000"] = round(entry["gbs"] / 8000.0, 3)
         kernels[name] = entry
     dom = "gemm1_swiglu"
     achieved = kernels[dom]["tflops"]
+    gemm_names = list(phase_flops)
+    nominal_fracs = {k: kernels[k]["frac_of_nominal_fp8_4500"] for k in gemm_names if k in kernels}
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": fp8_peak, "unit": "TFLOP/s",
                 "frac": round(achieved / fp8_peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                "peak_source": f"of {peak_kind}: 2 x bf16_tflops_sustained ({peaks['bf16_tflops_sustained']}) "
-                               "- no FP8 GEMM peak is measured on this pool, the nominal FP8:bf16 ratio is applied",
+                "peak_source": f"of {peak_kind}: 2 x bf16_tflops_sustained ({peaks['bf16_tflops_sustained']}), the measured "
+                               "bf16 rate of this pool times the nominal FP8:bf16 ratio; the FP8 rate measured in this "
+                               "very run is under measured_fp8_gemm",
+                "target_60pct_of_nominal_fp8": {
+                    "target_tflops": 0.6 * NOMINAL_FP8_TFLOPS, "nominal_tflops": NOMINAL_FP8_TFLOPS,
+                    "frac_of_nominal": nominal_fracs, "step_frac_of_nominal": round(value / world / NOMINAL_FP8_TFLOPS, 4),
+                    "met": {k: v >= 0.6 for k, v in nominal_fracs.items()},
+                    "why": "the board's power cap holds the SM clock well below its maximum during a sustained step "
+                           "(clocks.sm_mhz against clocks.sm_max_mhz; kernels.*.tflops_if_clock_held_at_max is the same "
+                           "cycle count at the maximum clock)"},
                 "frac_of_nominal_fp8_4500": round(achieved / NOMINAL_FP8_TFLOPS, 4),
+                "measured_fp8_gemm": vendor,
+                "frac_of_measured_fp8": kernels[dom].get("frac_of_measured_fp8"),
                 "algorithmic_flops_per_launch": phase_flops[dom],
                 "algorithmic_bytes_per_launch": float(T) * d + 2.0 * d * f + float(T) * f + 4.0 * T * f,
                 "step_frac_of_peak": round(value / world / fp8_peak, 4),
@@ -452,16 +672,19 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     d2h = 2 * T * d * 2
     out = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "ms_per_step_median": round(ms_median, 4),
+        "value_at_median_step": round(job_tflops(T, d, f, world, ms_median), 2), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "fp8 (E4M3 fwd / E5M2 grads, fp32 accumulate)", "data": "synthetic",
         "config": {"workload": args.workload, "T": T, "d_model": d, "d_ff": f, "smooth_swiglu": True,
-                   "scale_mode": "given (delayed), maxima emitted every step", "replicas": world,
+                   "scale_mode": "given (delayed): maxima emitted and turned into the next step's scales every step",
+                   "replicas": world,
                    "l2": "inputs per step (fp32 master weights 541 MB at the 7B shape) exceed the 126 MB L2"},
         "clocks": clocks,
         "e2e": {"value": round(job_tflops(T, d, f, world, e2e_ms), 2), "unit": UNIT,
                 "ms_per_step": round(e2e_ms, 4), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "what": "every step: x and dY copied from pinned host memory, Y and dX copied back to it; copies "
-                        "on their own streams overlap the neighbouring steps' kernels; weights resident"},
+                        "on their own streams overlap the neighbouring steps' kernels; the fp32 master weights and "
+                        "the 541 MB of weight gradients stay on the device, where the optimizer step consumes them"},
         "gpu_launches": launches,
         "roofline": roofline,
         "kernels": kernels,
@@ -484,15 +707,21 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     print(json.dumps(out))
 
 
+def wl_has_gradient(name: str) -> bool:
+    from paper_2409_12517_b200 import workloads as wl
+    return wl.CONFIGS[name].get("with_dy", True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-after-idle", action="store_true", help="skip the single steps timed after a second of idle")
+    ap.add_argument("--no-vendor-gemm", action="store_true", help="skip the vendor FP8 GEMM yardstick (about 15 s)")
     ap.add_argument("--ref-seconds", type=float, default=120.0,
                     help="--impl reference: CPU time the whole run may take (sizes the channel sample)")
     args = ap.parse_args()
@@ -502,6 +731,8 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+    elif not wl_has_gradient(args.workload):
+        run_forward_only(args, rank, local_rank)
     else:
         run_ours(args, rank, world, local_rank)
 
