@@ -211,7 +211,9 @@ FP8MLP_API int fp8mlp_forward_merged(fp8mlp_ctx* ctx, int64_t T, const void* x_b
  * the update divides by the square root of the second moment, so its smallest values matter and it
  * needs the wider exponent range).  The step after fp8mlp_backward: it consumes dW1, dW2, dW3.
  * The update is the textbook one (bias-corrected Adam, decoupled weight decay); per parameter i,
- * in fp32, one rounding per operation in this order:
+ * in fp32 in this order - the moments, codes and maxima with one rounding per operation (they are
+ * bit-exact against a plain CPU evaluation); the square root and the division of `upd` run on the
+ * special-function unit and are approximate to a few 2^-23 relative, which reaches only w:
  *   m_prev = dec_e4m3(m[i]) * (1 / *scale_m_in);     v_prev = dec_e5m2(v[i]) * (1 / *scale_v_in)
  *   mi = beta1 * m_prev + (1 - beta1) * g[i];        vi = beta2 * v_prev + (1 - beta2) * (g[i] * g[i])
  *   upd = (mi * c1) / (sqrt(vi * c2) + eps) [+ weight_decay * w[i]],   c = 1 / (1 - beta^step) (fp64, rounded once)
@@ -260,8 +262,10 @@ FP8MLP_API int fp8mlp_scale_from_amax(const float* amax, int fp8_fmt, float* sca
  * Arguments are those of fp8mlp_forward, with the shape and `flags` (FP8MLP_SMOOTH or 0) passed
  * directly instead of a context.  The caller still owns x, the weights, y, `scales` and `amax`.
  * It calls no cudaMalloc / cudaFree and no allocating library routine.
- *   - The first call on each device looks up the array's device address (once per device, with that
- *     device current).  Make that first call outside any stream capture.
+ *   - Every call asks the runtime for the array's address on the current device (the array exists once
+ *     per GPU; the device that is current at the call is the one used).  The first call on a device is
+ *     the one that makes the runtime set the array up there: make that first call outside any stream
+ *     capture.  Argument errors are found before the lookup and before anything is enqueued.
  *   - All calls share the one array, and it keeps whatever the previous call left in it; each call
  *     rewrites or clears everything it reads (the status word and the maxima start from zero).
  *     Two calls that overlap on the GPU (different streams, or different host threads without

@@ -145,7 +145,7 @@ GemmArgs base_args(fp8mlp_ctx* c, int M, int N, int K) {
     a.M = M; a.N = N; a.K = K;
     a.n_tile_cols = kBlockN;
     a.b1_offset = 128;
-    a.group_m = 16;
+    a.group = 16;
     a.status = c ? c->status : nullptr;
     a.n_split = N;
     a.ld_out = N;
@@ -196,6 +196,24 @@ int gemm1_swiglu(fp8mlp_ctx* c, int64_t T, const fp8mlp_scales* s, float* amax_h
     }
     a.amax_h = reinterpret_cast<unsigned int*>(amax_h);
     return launch_gemm(EPI_SWIGLU_FWD, false, true, FP8MLP_E4M3, FP8MLP_E4M3, tmA, tmB0, tmB1, a, c->sm_count, st);
+}
+
+// Everything fp8mlp_forward can refuse before it enqueues anything.
+int check_forward_args(const fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, const float* W2, const float* W3,
+                       int mode, const fp8mlp_scales* sc, const fp8mlp_amax* am, const void* y) {
+    if (c == nullptr || sc == nullptr || W1 == nullptr || W2 == nullptr || W3 == nullptr) return FP8MLP_ERR_ARG;
+    if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
+    if (!on_device_of(c)) return FP8MLP_ERR_STATE;
+    if (T < 0 || T > c->T_max) return FP8MLP_ERR_SHAPE;
+    if (T > 0 && (x == nullptr || y == nullptr)) return FP8MLP_ERR_ARG;
+    if (sc->x == nullptr || sc->w12 == nullptr || sc->w3 == nullptr || sc->h == nullptr) return FP8MLP_ERR_ARG;
+    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX &&
+        (am == nullptr || am->x == nullptr || am->w1 == nullptr || am->w2 == nullptr || am->w3 == nullptr || am->h == nullptr))
+        return FP8MLP_ERR_ARG;
+    const bool gu_fp8 = (c->flags & FP8MLP_GU_FP8) != 0;
+    if (gu_fp8 && (sc->gu == nullptr || (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX && am->gu == nullptr))) return FP8MLP_ERR_ARG;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(W1) || !aligned16(W2) || !aligned16(W3)) return FP8MLP_ERR_ALIGN;
+    return FP8MLP_OK;
 }
 
 }  // namespace
@@ -385,18 +403,8 @@ int fp8mlp_update_scales(fp8mlp_ctx* c, const fp8mlp_amax* am, fp8mlp_scales* sc
 
 int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, const float* W2, const float* W3,
                    int mode, fp8mlp_scales* sc, fp8mlp_amax* am, void* y, void* stream) {
-    if (c == nullptr || sc == nullptr || W1 == nullptr || W2 == nullptr || W3 == nullptr) return FP8MLP_ERR_ARG;
-    if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
-    if (!on_device_of(c)) return FP8MLP_ERR_STATE;
-    if (T < 0 || T > c->T_max) return FP8MLP_ERR_SHAPE;
-    if (T > 0 && (x == nullptr || y == nullptr)) return FP8MLP_ERR_ARG;
-    if (sc->x == nullptr || sc->w12 == nullptr || sc->w3 == nullptr || sc->h == nullptr) return FP8MLP_ERR_ARG;
-    if (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX &&
-        (am == nullptr || am->x == nullptr || am->w1 == nullptr || am->w2 == nullptr || am->w3 == nullptr || am->h == nullptr))
-        return FP8MLP_ERR_ARG;
+    FP8MLP_TRY(check_forward_args(c, T, x, W1, W2, W3, mode, sc, am, y));
     const bool gu_fp8 = (c->flags & FP8MLP_GU_FP8) != 0;
-    if (gu_fp8 && (sc->gu == nullptr || (mode == FP8MLP_SCALE_FROM_CURRENT_AMAX && am->gu == nullptr))) return FP8MLP_ERR_ARG;
-    if (!aligned16(x) || !aligned16(y) || !aligned16(W1) || !aligned16(W2) || !aligned16(W3)) return FP8MLP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool smooth = (c->flags & FP8MLP_SMOOTH) != 0;
     const int64_t d = c->d, f = c->f;
@@ -698,10 +706,10 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
 
 namespace {
 // Built-in scratch of fp8mlp_forward_static.  In host code this name is only a stand-in for the
-// symbol: the device address is looked up once per device with cudaGetSymbolAddress.
+// symbol, not a device address: the address on the current device is asked of the runtime with
+// cudaGetSymbolAddress (a table lookup after the first call on a device; asking every time keeps
+// no pointer that a cudaDeviceReset could leave stale).
 __device__ __align__(256) unsigned char g_static_scratch[FP8MLP_STATIC_SCRATCH_BYTES];
-constexpr int kMaxDevices = 64;
-unsigned char* g_static_scratch_ptr[kMaxDevices] = {};   // per device, filled on first use
 
 int64_t round_up_256(int64_t v) { return (v + 255) & ~int64_t(255); }
 }  // namespace
@@ -718,19 +726,18 @@ int fp8mlp_forward_static(int64_t T, int64_t d, int64_t f, uint32_t flags, const
 
     int dev = 0, sms = 0;
     FP8MLP_CUDA_CHECK(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= kMaxDevices) return FP8MLP_ERR_ARG;
-    if (g_static_scratch_ptr[dev] == nullptr) {
-        void* p = nullptr;
-        FP8MLP_CUDA_CHECK(cudaGetSymbolAddress(&p, g_static_scratch));
-        g_static_scratch_ptr[dev] = static_cast<unsigned char*>(p);
-    }
     FP8MLP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
 
-    // a context that lives on this stack frame and points into the built-in array
+    // a context that lives on this stack frame; its buffers are carved out of the built-in array below
     fp8mlp_ctx c;
     std::memset(&c, 0, sizeof(c));
     c.T_max = T; c.d = d; c.f = f; c.flags = flags; c.device = dev; c.sm_count = sms; c.saved_T = -1;
-    unsigned char* base = g_static_scratch_ptr[dev];
+    // every argument error is found here, before anything is enqueued
+    FP8MLP_TRY(check_forward_args(&c, T, x, W1, W2, W3, mode, sc, am, y));
+
+    void* sym = nullptr;
+    FP8MLP_CUDA_CHECK(cudaGetSymbolAddress(&sym, g_static_scratch));
+    unsigned char* base = static_cast<unsigned char*>(sym);
     int64_t off = 0;
     auto carve = [&](int64_t bytes) { unsigned char* p = base + off; off += round_up_256(bytes); return p; };
     c.status = reinterpret_cast<int*>(carve(256));

@@ -64,28 +64,44 @@ __device__ __forceinline__ uint32_t k_step_bytes() { return MN_MAJOR ? (32u / EL
 // One operand block of 128 rows x 128 bytes of K into shared memory (16 KiB): a K-major operand is
 // one TMA box; an MN-major operand is ELEM boxes of 128 / ELEM rows each, side by side.
 template <bool MN_MAJOR, int ELEM, bool PAIR>
-__device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row0, int k0) {
+__device__ __forceinline__ void load_operand(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row0, int k0, int hint,
+                                             uint64_t policy) {
+    auto box = [&](uint32_t to, int x, int y) {
+        if (hint == L2_HINT_NONE) {
+            if constexpr (PAIR) tma_load_2d_pair(to, map, bar, x, y); else tma_load_2d(to, map, bar, x, y);
+        } else {
+            if constexpr (PAIR) tma_load_2d_pair_hint(to, map, bar, x, y, policy); else tma_load_2d_hint(to, map, bar, x, y, policy);
+        }
+    };
     if constexpr (!MN_MAJOR) {
-        if constexpr (PAIR) tma_load_2d_pair(dst, map, bar, k0, row0); else tma_load_2d(dst, map, bar, k0, row0);
+        box(dst, k0, row0);
     } else {
 #pragma unroll
-        for (int h = 0; h < ELEM; ++h) {
-            if constexpr (PAIR) tma_load_2d_pair(dst + h * (kBoxBytes / ELEM), map, bar, row0 + h * (128 / ELEM), k0);
-            else tma_load_2d(dst + h * (kBoxBytes / ELEM), map, bar, row0 + h * (128 / ELEM), k0);
-        }
+        for (int h = 0; h < ELEM; ++h) box(dst + h * (kBoxBytes / ELEM), row0 + h * (128 / ELEM), k0);
     }
 }
 
 __device__ __forceinline__ void tile_coords(const GemmArgs& p, int tile, int& m_tile, int& n_tile) {
-    // bands of group_m m-tiles; inside a band consecutive tiles walk down m first, so the CTAs
-    // running at the same time share a few A row-blocks and a few B column-blocks in L2
-    const int per_band = p.group_m * p.num_n_tiles;
-    const int band = tile / per_band;
-    const int first_m = band * p.group_m;
-    const int rows = min(p.num_m_tiles - first_m, p.group_m);
-    const int in_band = tile - band * per_band;
-    m_tile = first_m + in_band % rows;
-    n_tile = in_band / rows;
+    // Bands of `group` tiles along one dimension, walked along that dimension first, so that the CTAs running at
+    // the same time share a few A row-blocks and a few B column-blocks in L2.  The band's slice of the operand
+    // indexed by the banded dimension is what every wave of the band reads again.
+    if (p.band_n == 0) {                 // bands of group m-tiles; the band's A rows are re-read
+        const int per_band = p.group * p.num_n_tiles;
+        const int band = tile / per_band;
+        const int first_m = band * p.group;
+        const int rows = min(p.num_m_tiles - first_m, p.group);
+        const int in_band = tile - band * per_band;
+        m_tile = first_m + in_band % rows;
+        n_tile = in_band / rows;
+    } else {                             // bands of group n-tiles; the band's B rows are re-read
+        const int per_band = p.group * p.num_m_tiles;
+        const int band = tile / per_band;
+        const int first_n = band * p.group;
+        const int cols = min(p.num_n_tiles - first_n, p.group);
+        const int in_band = tile - band * per_band;
+        n_tile = first_n + in_band % cols;
+        m_tile = in_band / cols;
+    }
 }
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
@@ -303,8 +319,12 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
         const uint32_t slot = gu_count % kGuSlots, phase = (gu_count / kGuSlots) & 1u;
         const int col = 64 * c + 32 * half;            // first of this warp's 32 accumulator columns
         const int c0 = n0 + col;
-        if (!gu8 || (c & 1) == 0)                      // codes: the slot of chunk c - 1 also holds chunk c
-            if (!mbar_wait(smem_u32(&tail->gu_full[slot]), phase, abort_flag, p.status)) return false;
+        if (!gu8 || (c & 1) == 0) {                    // codes: the slot of chunk c - 1 also holds chunk c
+            // the warp leaves together or not at all: a wait that ran out for some lanes only would split it
+            // between the failure path and the warp-wide instructions below
+            const bool landed = mbar_wait(smem_u32(&tail->gu_full[slot]), phase, abort_flag, p.status);
+            if (!__all_sync(0xffffffffu, landed)) return false;
+        }
         uint4 gq[4], uq[4];
         {
             const uint32_t rbase = gu_base + slot * kGuSlotBytes + static_cast<uint32_t>(row) * 128u;
@@ -465,6 +485,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             const CUtensorMap* tmB = (PAIR && rank != 0) ? &tmB1 : &tmB0;
+            const uint64_t pol_a = l2_policy(p.hint_a), pol_b = l2_policy(p.hint_b);
             for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
                 int m_tile, n_tile;
                 tile_coords(p, tile, m_tile, n_tile);
@@ -479,15 +500,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         // both CTAs' bytes are counted on rank 0's barrier, armed by rank 0 for both
                         const uint32_t bar = mapa_shared(smem_u32(&tail->full[stage]), 0);
                         if (rank == 0) mbar_expect_tx(smem_u32(&tail->full[stage]), 2 * kStageBytes);
-                        load_operand<A_MN, ELEM, true>(dst, &tmA, bar, m0, k0);
-                        load_operand<B_MN, ELEM, true>(dst + kBoxBytes, tmB, bar, nb0, k0);
-                        if constexpr (WIDEN) load_operand<B_MN, ELEM, true>(dst + 2 * kBoxBytes, tmB, bar, nb0 + kBlockN, k0);
+                        load_operand<A_MN, ELEM, true>(dst, &tmA, bar, m0, k0, p.hint_a, pol_a);
+                        load_operand<B_MN, ELEM, true>(dst + kBoxBytes, tmB, bar, nb0, k0, p.hint_b, pol_b);
+                        if constexpr (WIDEN) load_operand<B_MN, ELEM, true>(dst + 2 * kBoxBytes, tmB, bar, nb0 + kBlockN, k0, p.hint_b, pol_b);
                     } else {
                         const uint32_t bar = smem_u32(&tail->full[stage]);
                         mbar_expect_tx(bar, kStageBytes);
-                        load_operand<A_MN, ELEM, false>(dst, &tmA, bar, m0, k0);
-                        load_operand<B_MN, ELEM, false>(dst + kBoxBytes, &tmB0, bar, nb0, k0);
-                        load_operand<B_MN, ELEM, false>(dst + 2 * kBoxBytes, &tmB1, bar, nb1, k0);
+                        load_operand<A_MN, ELEM, false>(dst, &tmA, bar, m0, k0, p.hint_a, pol_a);
+                        load_operand<B_MN, ELEM, false>(dst + kBoxBytes, &tmB0, bar, nb0, k0, p.hint_b, pol_b);
+                        load_operand<B_MN, ELEM, false>(dst + 2 * kBoxBytes, &tmB1, bar, nb1, k0, p.hint_b, pol_b);
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
@@ -784,7 +805,7 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     const int elem = args.elem_bytes == 2 ? 2 : 1;
     const int kblk = kBlockK / elem;     // contraction elements per stage
     args.num_k_blocks = (args.K + kblk - 1) / kblk;
-    if (args.group_m <= 0) args.group_m = pair ? 8 : 16;
+    if (args.group <= 0) args.group = pair ? 8 : 16;
     // instruction descriptor: [4,6) D = fp32; [7,10) A format; [10,13) B format (0 = E4M3, 1 = E5M2);
     // bit 15 / 16: A / B is MN-major; [17,23) N >> 3; [24,29) M >> 4 (M counts both CTAs of a pair)
     args.idesc = (1u << 4) | (static_cast<uint32_t>(a_fmt) << 7) | (static_cast<uint32_t>(b_fmt) << 10) |

@@ -42,7 +42,9 @@ struct GemmArgs {
     int num_m_tiles, num_n_tiles, num_k_blocks;
     int n_tile_cols;        // n coordinates per tile: 256, or 128 when the two B boxes are gate and linear halves
     int b1_offset;          // n offset of the second B box: 128, or 0 in the gate/linear case
-    int group_m;            // m-tiles per rasterisation band
+    int group;              // tiles per rasterisation band, counted along m (band_n = 0) or along n (band_n = 1)
+    int band_n;
+    int hint_a, hint_b;     // L2 eviction priority of the A / B operand loads (L2_HINT_*)
     int pair_mode;          // 0: CTA pairs when M > 128; 1: always CTA pairs; 2: always single CTAs
     int elem_bytes;         // operand element size: 1 (FP8, default) or 2 (bf16; a_fmt = b_fmt = 1)
     int wide_tiles;         // 256 x 512 tiles: 0 = for bf16 outputs (default), 1 = for fp32 outputs too, 2 = never
