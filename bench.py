@@ -542,6 +542,43 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         adam_bytes = 16.0 * 3 * d * f                # g 4 + w 4+4 + codes 1+1+1+1 per parameter
         adam = {"ms": round(adam_ms, 4), "params": 3 * d * f, "bytes_per_param": 16,
                 "gbs": round(adam_bytes / (adam_ms * 1e-3) / 1e9, 1)}
+        # The training step including its optimizer step, two ways: the weight cast inside the next forward (as in
+        # `value`), or fused into the Adam pass, which reads and writes every master weight anyway (the next forward
+        # then takes the FP8 weights as they are).  Same work either way; neither is `value`.
+        p12, _ = B.fp8mlp_workspace(ctx, B.WS_W12Q)
+        p3, _ = B.fp8mlp_workspace(ctx, B.WS_W3Q)
+        casts = [dict(dst=p12 + f, cols=f, ld_dst=2 * f, scale=sc["w12"], amax=am["w1"]),
+                 dict(dst=p12, cols=f, ld_dst=2 * f, scale=sc["w12"], amax=am["w2"]),
+                 dict(dst=p3, cols=d, ld_dst=d, scale=sc["w3"], row_div=sc["h"], amax=am["w3"])]
+
+        def train_plain(t):
+            step()
+            B.fp8mlp_adam_step(states, step=t, **hp)
+
+        def train_fused(t):
+            B.fp8mlp_forward(ctx, T, x, None, None, None, B.SCALE_GIVEN_WEIGHTS_CAST, sc, am, y)
+            B.fp8mlp_backward(ctx, T, dy, B.SCALE_GIVEN, sc, am, dx, dW1, dW2, dW3)
+            B.fp8mlp_update_scales(ctx, am, sc)
+            B.fp8mlp_adam_step_cast(states, casts, step=t, **hp)
+
+        fused = {}
+        n_tr = max(1, min(args.steps, 50))
+        for name, fn in (("cast_in_forward", train_plain), ("cast_fused_into_adam", train_fused)):
+            if name == "cast_fused_into_adam":
+                B.fp8mlp_adam_step_cast(states, casts, step=100, **hp)      # the first fused forward needs codes to start from
+            for t in range(3):
+                fn(101 + t)
+            torch.cuda.synchronize()
+            e0.record()
+            for t in range(n_tr):
+                fn(110 + t)
+            e1.record()
+            torch.cuda.synchronize()
+            fused[name + "_ms"] = round(e0.elapsed_time(e1) / n_tr, 4)
+        assert B.fp8mlp_status(ctx) == B.OK
+        fused["what"] = "forward + backward + scale update + Adam step with FP8 moments, per training step"
+        adam["training_step_with_optimizer"] = fused
+        step()                                        # leaves the context's weight codes and scales as the step makes them
         del states
     # the same step with every scale derived just in time (extra amax passes, GEMM-1 and dgrad-2 run twice)
     jit = None

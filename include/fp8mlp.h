@@ -65,7 +65,10 @@ enum {
 };
 enum {
     FP8MLP_SCALE_GIVEN = 0,              /* delayed scaling: use the scale buffers as they are  */
-    FP8MLP_SCALE_FROM_CURRENT_AMAX = 1   /* just-in-time: derive every scale from this call's data */
+    FP8MLP_SCALE_FROM_CURRENT_AMAX = 1,  /* just-in-time: derive every scale from this call's data */
+    FP8MLP_SCALE_GIVEN_WEIGHTS_CAST = 2  /* fp8mlp_forward only: as SCALE_GIVEN, and the context's FP8 weight buffers
+                                            already hold this step's codes (fp8mlp_adam_step_cast wrote them): the
+                                            weight pass is skipped, W1/W2/W3 are not read (may be null), amax.w* stay */
 };
 enum { /* fp8mlp_workspace: internal buffers, for inspection by tests */
     FP8MLP_WS_XQ = 0,   /* E4M3 [T,d]   quantised x                                   */
@@ -241,6 +244,28 @@ typedef struct {
 } fp8mlp_adam_tensor;
 FP8MLP_API int fp8mlp_adam_step(const fp8mlp_adam_tensor* tensors, int count, float lr, float beta1, float beta2,
                                 float eps, float weight_decay, int64_t step, void* stream);
+/* The same step, which also casts the updated master weights to the E4M3 operands of the next forward
+ * (Section 6.2: high-precision master weights, quantised to E4M3 for the forward phase): the pass already reads
+ * and writes every weight, so the cast costs one more byte written per parameter instead of a pass of its own
+ * (4 bytes read + 1 written).  Per tensor i, casts[i] describes the codes (dst = null: none for this tensor):
+ *   the tensor is a [n / cols, cols] matrix; code[r, c] = Q_e4m3((w_new[r, c] / row_div[r]) * *scale) at
+ *   dst[r * ld_dst + c]; *amax = max |w_new[r, c] / row_div[r]|   (row_div nullable = no division; the
+ *   division is a multiplication by the fp32 reciprocal, as in the forward's own quantise pass).
+ * With dst pointing into the context's FP8 weight buffers (fp8mlp_workspace: W1 at FP8MLP_WS_W12Q + d_ff with
+ * ld_dst = 2 d_ff, W2 at FP8MLP_WS_W12Q with ld_dst = 2 d_ff, both with scales.w12; W3 at FP8MLP_WS_W3Q with
+ * scales.w3 and row_div = scales.h for Smooth-SwiGLU) the next fp8mlp_forward can be called with
+ * FP8MLP_SCALE_GIVEN_WEIGHTS_CAST and skips its weight pass.  cols, ld_dst multiples of 16; dst 16-byte aligned. */
+typedef struct {
+    uint8_t* dst;              /* [n / cols, ld_dst] E4M3 codes, or null         */
+    int64_t cols;
+    int64_t ld_dst;
+    const float* scale;        /* device float                                   */
+    const float* row_div;      /* device [n / cols], nullable                    */
+    float* amax;               /* device float out, nullable                     */
+} fp8mlp_adam_cast;
+FP8MLP_API int fp8mlp_adam_step_cast(const fp8mlp_adam_tensor* tensors, const fp8mlp_adam_cast* casts, int count,
+                                     float lr, float beta1, float beta2, float eps, float weight_decay, int64_t step,
+                                     void* stream);
 /* *scale = fmt_max / *amax (Section 2, per-tensor scaling; 1 if *amax is zero or not finite).
  * fp8_fmt FP8MLP_E4M3 or FP8MLP_E5M2; both pointers device floats. */
 FP8MLP_API int fp8mlp_scale_from_amax(const float* amax, int fp8_fmt, float* scale, void* stream);

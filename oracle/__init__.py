@@ -322,3 +322,14 @@ def adam_step(w, g, mq, vq, *, lr, beta1, beta2, eps, weight_decay, step, sm_in=
                           C.c_int64(step), C.c_float(sm_in), C.c_float(sv_in), C.c_float(sm_out), C.c_float(sv_out),
                           C.byref(am), C.byref(av))
     return float(am.value), float(av.value)
+
+
+def adam_step_and_cast(w, g, mq, vq, *, cols: int, scale: float, row_div=None, **adam):
+    """The optimizer step followed by the E4M3 cast of the updated master weights for the next forward (Section 6.2
+    of the paper keeps high-precision master weights and quantises them to E4M3 for the forward phase): the
+    composition adam_step -> quantize of this module, nothing else.  w is updated in place; returns
+    (amax_m, amax_v, codes [n / cols, cols], amax of the cast values)."""
+    am, av = adam_step(w, g, mq, vq, **adam)
+    inv = None if row_div is None else (np.float32(1.0) / np.asarray(row_div, np.float32)).astype(np.float32)
+    codes, _, amax_w = quantize(w.reshape(-1, cols), E4M3, scale, row_mul=inv)
+    return am, av, codes, amax_w

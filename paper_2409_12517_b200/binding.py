@@ -20,7 +20,7 @@ STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 E4M3, E5M2 = 0, 1
 BF16, F32 = 0, 1
 SMOOTH, SAVE_FOR_BWD, H_BF16, GU_FP8 = 1, 2, 4, 8
-SCALE_GIVEN, SCALE_FROM_CURRENT_AMAX = 0, 1
+SCALE_GIVEN, SCALE_FROM_CURRENT_AMAX, SCALE_GIVEN_WEIGHTS_CAST = 0, 1, 2
 WS_XQ, WS_W12Q, WS_W3Q, WS_HQ, WS_GU, WS_DYQ, WS_DZQ, WS_HB, WS_W3B = range(9)
 
 EXPORTS = [
@@ -29,7 +29,7 @@ EXPORTS = [
     "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8", "fp8mlp_profile_enable", "fp8mlp_profile_read",
     "fp8mlp_forward_static", "fp8mlp_adam_step", "fp8mlp_scale_from_amax",
     "fp8mlp_merge_weights", "fp8mlp_forward_merged", "fp8mlp_gemm_bf16",
-    "fp8mlp_selftest_wait_timeout",
+    "fp8mlp_selftest_wait_timeout", "fp8mlp_adam_step_cast",
 ]
 PHASES = ["quant_x", "quant_w12", "quant_w3", "gemm1_swiglu", "gemm2_down", "quant_dy", "dgrad2_swiglu_bwd",
           "wgrad3", "dgrad1", "wgrad12", "misc"]
@@ -55,6 +55,11 @@ class _AdamTensor(C.Structure):
     _fields_ = [("w", C.c_void_p), ("g", C.c_void_p), ("m", C.c_void_p), ("v", C.c_void_p), ("n", C.c_int64),
                 ("scale_m_in", C.c_void_p), ("scale_v_in", C.c_void_p), ("scale_m_out", C.c_void_p),
                 ("scale_v_out", C.c_void_p), ("amax_m", C.c_void_p), ("amax_v", C.c_void_p)]
+
+
+class _AdamCast(C.Structure):
+    _fields_ = [("dst", C.c_void_p), ("cols", C.c_int64), ("ld_dst", C.c_int64), ("scale", C.c_void_p),
+                ("row_div", C.c_void_p), ("amax", C.c_void_p)]
 
 
 _lib = None
@@ -97,6 +102,8 @@ def lib():
                                             C.POINTER(_Amax), C.c_void_p, C.c_void_p]
         L.fp8mlp_adam_step.argtypes = [C.POINTER(_AdamTensor), C.c_int, C.c_float, C.c_float, C.c_float, C.c_float,
                                        C.c_float, C.c_int64, C.c_void_p]
+        L.fp8mlp_adam_step_cast.argtypes = [C.POINTER(_AdamTensor), C.POINTER(_AdamCast), C.c_int, C.c_float, C.c_float,
+                                            C.c_float, C.c_float, C.c_float, C.c_int64, C.c_void_p]
         L.fp8mlp_scale_from_amax.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         L.fp8mlp_profile_enable.argtypes = [C.c_void_p, C.c_int]
         L.fp8mlp_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -243,6 +250,28 @@ def fp8mlp_adam_step(tensors: list, lr: float, beta1: float, beta2: float, eps: 
             setattr(a, k, t[k].data_ptr())
     _check(lib().fp8mlp_adam_step(arr, len(tensors), lr, beta1, beta2, eps, weight_decay, step, _stream()),
            "fp8mlp_adam_step")
+
+
+def fp8mlp_adam_step_cast(tensors: list, casts: list, lr: float, beta1: float, beta2: float, eps: float,
+                          weight_decay: float, step: int) -> None:
+    """fp8mlp_adam_step that also writes the E4M3 codes of the updated weights.  casts: one entry per tensor, None or a
+    dict with dst (device pointer as int, or a uint8 tensor), cols, ld_dst, scale (1-element fp32 tensor), and
+    optionally row_div (fp32 tensor, one per row) and amax (1-element fp32 tensor)."""
+    arr = (_AdamTensor * len(tensors))()
+    for a, t in zip(arr, tensors):
+        a.w, a.g, a.m, a.v, a.n = t["w"].data_ptr(), t["g"].data_ptr(), t["m"].data_ptr(), t["v"].data_ptr(), t["w"].numel()
+        for k in ("scale_m_in", "scale_v_in", "scale_m_out", "scale_v_out", "amax_m", "amax_v"):
+            setattr(a, k, t[k].data_ptr())
+    carr = (_AdamCast * len(tensors))()
+    for c, d in zip(carr, casts):
+        if d is None:
+            continue
+        c.dst = d["dst"] if isinstance(d["dst"], int) else d["dst"].data_ptr()
+        c.cols, c.ld_dst, c.scale = d["cols"], d["ld_dst"], d["scale"].data_ptr()
+        c.row_div = d["row_div"].data_ptr() if d.get("row_div") is not None else None
+        c.amax = d["amax"].data_ptr() if d.get("amax") is not None else None
+    _check(lib().fp8mlp_adam_step_cast(arr, carr, len(tensors), lr, beta1, beta2, eps, weight_decay, step, _stream()),
+           "fp8mlp_adam_step_cast")
 
 
 def fp8mlp_scale_from_amax(amax, fp8_fmt: int, scale) -> None:

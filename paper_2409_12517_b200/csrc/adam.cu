@@ -21,16 +21,20 @@ struct AdamSeg {
     const float *sm_in, *sv_in, *sm_out, *sv_out;
     float *amax_m, *amax_v;
     uint32_t n_units, units_per_block;     // a unit is 8 parameters
+    // optional cast of the updated weights to the E4M3 operand of the next forward
+    uint8_t* q_dst; int64_t q_ld; uint32_t q_units_per_row; const float* q_scale; const float* q_row_div; float* q_amax;
 };
 struct AdamLaunch {
     AdamSeg seg[kAdamMaxTensors];
     int nseg, wide;
     float lr, beta1, beta2, omb1, omb2, c1, c2, eps, wd;
 };
-struct AdamZero { float* p[2 * kAdamMaxTensors]; };
+struct AdamZero { float* p[3 * kAdamMaxTensors]; };
 
 __global__ void adam_zero_kernel(AdamZero z) {
-    if (threadIdx.x < 2 * kAdamMaxTensors && z.p[threadIdx.x] != nullptr) *z.p[threadIdx.x] = 0.0f;
+    grid_dependency_wait();
+    grid_launch_dependents();
+    if (threadIdx.x < 3 * kAdamMaxTensors && z.p[threadIdx.x] != nullptr) *z.p[threadIdx.x] = 0.0f;
 }
 
 // 8 FP8 codes (two 32-bit words) -> 8 floats, exactly
@@ -56,9 +60,17 @@ __device__ __forceinline__ float warp_max_f(float v) {
     return v;
 }
 
+// CAST: the pass also writes the E4M3 codes of the updated weights (scale, optional per-row divisor: exactly the
+// arithmetic of the quantise pass of the forward, which the next forward can then skip) and their maximum.
+template <bool CAST>
 __global__ void __launch_bounds__(kAdamThreads, kAdamBlocksPerSm) adam_kernel(const AdamLaunch q) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int seg_id = blockIdx.x % q.nseg;
     const AdamSeg& sg = q.seg[seg_id];
+    const bool cast = CAST && sg.q_dst != nullptr;
+    const float q_scale = cast ? *sg.q_scale : 1.0f;
+    float max_q = 0.0f;
     const uint32_t begin = (blockIdx.x / q.nseg) * sg.units_per_block;
     const uint32_t end = min(begin + sg.units_per_block, sg.n_units);
     const float inv_sm = __fdiv_rn(1.0f, *sg.sm_in), inv_sv = __fdiv_rn(1.0f, *sg.sv_in);
@@ -127,24 +139,44 @@ __global__ void __launch_bounds__(kAdamThreads, kAdamBlocksPerSm) adam_kernel(co
                 st_global_v4(sg.w + e0, wn[0], wn[1], wn[2], wn[3]);
                 st_global_v4(sg.w + e0 + 4, wn[4], wn[5], wn[6], wn[7]);
             }
+            if (CAST && cast) {
+                const uint32_t r = u / sg.q_units_per_row, cu = u - r * sg.q_units_per_row;
+                float t[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) t[i] = __uint_as_float(wn[i]);
+                if (sg.q_row_div != nullptr) {
+                    const float inv = __fdiv_rn(1.0f, sg.q_row_div[r]);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) t[i] = __fmul_rn(t[i], inv);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) max_q = fmaxf(max_q, fabsf(t[i]));
+                st_global_v2(sg.q_dst + static_cast<int64_t>(r) * sg.q_ld + static_cast<int64_t>(cu) * 8,
+                             cvt_fp8x4<FP8MLP_E4M3>(__fmul_rn(t[0], q_scale), __fmul_rn(t[1], q_scale), __fmul_rn(t[2], q_scale), __fmul_rn(t[3], q_scale)),
+                             cvt_fp8x4<FP8MLP_E4M3>(__fmul_rn(t[4], q_scale), __fmul_rn(t[5], q_scale), __fmul_rn(t[6], q_scale), __fmul_rn(t[7], q_scale)));
+            }
             st_global_v2(sg.m + e0, cvt_fp8x4<FP8MLP_E4M3>(ms[0], ms[1], ms[2], ms[3]), cvt_fp8x4<FP8MLP_E4M3>(ms[4], ms[5], ms[6], ms[7]));
             st_global_v2(sg.v + e0, cvt_fp8x4<FP8MLP_E5M2>(vs[0], vs[1], vs[2], vs[3]), cvt_fp8x4<FP8MLP_E5M2>(vs[4], vs[5], vs[6], vs[7]));
         }
     }
     // block-wide maxima (non-negative: their bit patterns order like unsigned integers)
-    __shared__ float part[2][kAdamThreads / 32];
+    __shared__ float part[3][kAdamThreads / 32];
     max_m = warp_max_f(max_m);
     max_v = warp_max_f(max_v);
-    if ((threadIdx.x & 31) == 0) { part[0][threadIdx.x >> 5] = max_m; part[1][threadIdx.x >> 5] = max_v; }
+    max_q = warp_max_f(max_q);
+    if ((threadIdx.x & 31) == 0) { part[0][threadIdx.x >> 5] = max_m; part[1][threadIdx.x >> 5] = max_v; part[2][threadIdx.x >> 5] = max_q; }
     __syncthreads();
     if (threadIdx.x < 32) {
         float a = threadIdx.x < kAdamThreads / 32 ? part[0][threadIdx.x] : 0.0f;
         float b = threadIdx.x < kAdamThreads / 32 ? part[1][threadIdx.x] : 0.0f;
+        float c = threadIdx.x < kAdamThreads / 32 ? part[2][threadIdx.x] : 0.0f;
         a = warp_max_f(a);
         b = warp_max_f(b);
+        c = warp_max_f(c);
         if (threadIdx.x == 0) {
             if (a > 0.0f) atomicMax(reinterpret_cast<unsigned int*>(sg.amax_m), __float_as_uint(a));
             if (b > 0.0f) atomicMax(reinterpret_cast<unsigned int*>(sg.amax_v), __float_as_uint(b));
+            if (CAST && cast && sg.q_amax != nullptr && c > 0.0f) atomicMax(reinterpret_cast<unsigned int*>(sg.q_amax), __float_as_uint(c));
         }
     }
 }
@@ -157,9 +189,17 @@ bool al(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (
 
 using namespace fp8mlp;
 
-extern "C" int fp8mlp_adam_step(const fp8mlp_adam_tensor* t, int count, float lr, float beta1, float beta2, float eps,
-                                float weight_decay, int64_t step, void* stream) {
+namespace {
+int adam_launch(const fp8mlp_adam_tensor* t, const fp8mlp_adam_cast* casts, int count, float lr, float beta1, float beta2,
+                float eps, float weight_decay, int64_t step, void* stream) {
     if (t == nullptr || count < 1 || count > kAdamMaxTensors) return FP8MLP_ERR_ARG;
+    for (int i = 0; casts != nullptr && i < count; ++i) {
+        const fp8mlp_adam_cast& c = casts[i];
+        if (c.dst == nullptr) continue;
+        if (c.scale == nullptr) return FP8MLP_ERR_ARG;
+        if (c.cols <= 0 || c.cols % 16 != 0 || c.ld_dst < c.cols || c.ld_dst % 16 != 0 || t[i].n % c.cols != 0) return FP8MLP_ERR_SHAPE;
+        if (!al(c.dst, 16)) return FP8MLP_ERR_ALIGN;
+    }
     if (step < 1 || !(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f)) return FP8MLP_ERR_ARG;
     int64_t worst = 0;
     for (int i = 0; i < count; ++i) {
@@ -177,8 +217,11 @@ extern "C" int fp8mlp_adam_step(const fp8mlp_adam_tensor* t, int count, float lr
     FP8MLP_CUDA_CHECK(cudaGetDevice(&dev));
     FP8MLP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     AdamZero z{};
-    for (int i = 0; i < count; ++i) { z.p[2 * i] = t[i].amax_m; z.p[2 * i + 1] = t[i].amax_v; }
-    adam_zero_kernel<<<1, 32, 0, st>>>(z);
+    for (int i = 0; i < count; ++i) {
+        z.p[3 * i] = t[i].amax_m; z.p[3 * i + 1] = t[i].amax_v;
+        z.p[3 * i + 2] = (casts != nullptr && casts[i].dst != nullptr) ? casts[i].amax : nullptr;
+    }
+    FP8MLP_CUDA_CHECK(launch_chained(adam_zero_kernel, 1, 32, 0, st, z));
     FP8MLP_LAUNCH_CHECK();
     if (worst == 0) return FP8MLP_OK;
 
@@ -204,8 +247,26 @@ extern "C" int fp8mlp_adam_step(const fp8mlp_adam_tensor* t, int count, float lr
         sg.n_units = static_cast<uint32_t>(t[i].n / 8);
         sg.units_per_block = static_cast<uint32_t>(((t[i].n / 8 + per_seg - 1) / per_seg + 31) / 32 * 32);
         if (!al(t[i].w, 32) || !al(t[i].g, 32)) q.wide = 0;
+        if (casts != nullptr && casts[i].dst != nullptr) {
+            sg.q_dst = casts[i].dst; sg.q_ld = casts[i].ld_dst; sg.q_units_per_row = static_cast<uint32_t>(casts[i].cols / 8);
+            sg.q_scale = casts[i].scale; sg.q_row_div = casts[i].row_div; sg.q_amax = casts[i].amax;
+        }
     }
-    adam_kernel<<<static_cast<int>(per_seg) * count, kAdamThreads, 0, st>>>(q);
+    const int grid = static_cast<int>(per_seg) * count;
+    if (casts != nullptr) FP8MLP_CUDA_CHECK(launch_chained(adam_kernel<true>, grid, kAdamThreads, 0, st, q));
+    else FP8MLP_CUDA_CHECK(launch_chained(adam_kernel<false>, grid, kAdamThreads, 0, st, q));
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
+}
+}  // namespace
+
+extern "C" int fp8mlp_adam_step(const fp8mlp_adam_tensor* t, int count, float lr, float beta1, float beta2, float eps,
+                                float weight_decay, int64_t step, void* stream) {
+    return adam_launch(t, nullptr, count, lr, beta1, beta2, eps, weight_decay, step, stream);
+}
+
+extern "C" int fp8mlp_adam_step_cast(const fp8mlp_adam_tensor* t, const fp8mlp_adam_cast* casts, int count, float lr,
+                                     float beta1, float beta2, float eps, float weight_decay, int64_t step, void* stream) {
+    if (casts == nullptr) return FP8MLP_ERR_ARG;
+    return adam_launch(t, casts, count, lr, beta1, beta2, eps, weight_decay, step, stream);
 }

@@ -25,9 +25,13 @@ void set_cuda_error_str(const char* what, const char* msg) {
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 // Sets up to 8 device floats and one vector of floats to zero in one launch (amax accumulators).
-struct ZeroList { float* p[8]; float* vec; int64_t n; };
+struct ZeroList { float* p[8]; float* vec; int64_t n; unsigned int* words; int n_words; };
 __global__ void zero_floats_kernel(ZeroList z) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     if (blockIdx.x == 0 && threadIdx.x < 8 && z.p[threadIdx.x] != nullptr) *z.p[threadIdx.x] = 0.0f;
+    if (blockIdx.x == 0)        // the split-contraction counters (a kernel that gave up on a wait may have left some set)
+        for (int i = threadIdx.x; i < z.n_words; i += blockDim.x) z.words[i] = 0u;
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < z.n;
          i += static_cast<int64_t>(gridDim.x) * blockDim.x)
         z.vec[i] = 0.0f;
@@ -58,6 +62,8 @@ struct fp8mlp_ctx {
     uint8_t *xq, *w12q, *w3q, *hq, *dyq, *dzq;
     uint16_t* gu;
     uint16_t *hb, *w3b;  // FP8MLP_H_BF16: the SwiGLU output and W3 in bf16 (operands of the unquantised last layer)
+    float* splitk_ws;           // fp32 partial tiles of a split contraction (small problems), kSplitFloats of them
+    unsigned int* splitk_cnt;   // their arrival counters, kSplitWords words
     float* dummy;     // [8 + f] sinks for amax outputs the caller did not ask for
     int* status;      // bounded-wait status word
     int64_t saved_T;  // tokens of the last forward that saved activations, -1 if none
@@ -106,14 +112,20 @@ bool on_device_of(const fp8mlp_ctx* c) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int zero_floats(std::initializer_list<float*> ptrs, cudaStream_t st, float* vec = nullptr, int64_t n_vec = 0) {
+// A split contraction is only made when the problem has fewer tiles than the device has CTA pairs, so its shares
+// number at most that many 256 x 256 tiles; 128 pairs cover every device this library runs on.
+constexpr int64_t kSplitFloats = int64_t(128) * 256 * 256;
+constexpr int kSplitWords = 128 * 16;
+
+int zero_floats(const fp8mlp_ctx* c, std::initializer_list<float*> ptrs, cudaStream_t st, float* vec = nullptr, int64_t n_vec = 0) {
     ZeroList z{};
     int n = 0;
     for (float* p : ptrs) z.p[n++] = p;
     z.vec = vec;
     z.n = vec != nullptr ? n_vec : 0;
+    if (c != nullptr && c->splitk_cnt != nullptr) { z.words = c->splitk_cnt; z.n_words = kSplitWords; }
     const int blocks = z.n > 256 ? static_cast<int>((z.n + 255) / 256 < 256 ? (z.n + 255) / 256 : 256) : 1;
-    zero_floats_kernel<<<blocks, 256, 0, st>>>(z);
+    FP8MLP_CUDA_CHECK(launch_chained(zero_floats_kernel, blocks, 256, 0, st, z));
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
 }
@@ -145,8 +157,11 @@ GemmArgs base_args(fp8mlp_ctx* c, int M, int N, int K) {
     a.M = M; a.N = N; a.K = K;
     a.n_tile_cols = kBlockN;
     a.b1_offset = 128;
-    a.group = 16;
     a.status = c ? c->status : nullptr;
+    if (c != nullptr && c->splitk_ws != nullptr && c->splitk_cnt != nullptr) {
+        a.partial = c->splitk_ws; a.partial_floats = kSplitFloats;
+        a.tile_counters = c->splitk_cnt; a.counter_words = kSplitWords;
+    }
     a.n_split = N;
     a.ld_out = N;
     a.store = 1;
@@ -201,8 +216,11 @@ int gemm1_swiglu(fp8mlp_ctx* c, int64_t T, const fp8mlp_scales* s, float* amax_h
 // Everything fp8mlp_forward can refuse before it enqueues anything.
 int check_forward_args(const fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, const float* W2, const float* W3,
                        int mode, const fp8mlp_scales* sc, const fp8mlp_amax* am, const void* y) {
-    if (c == nullptr || sc == nullptr || W1 == nullptr || W2 == nullptr || W3 == nullptr) return FP8MLP_ERR_ARG;
-    if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX) return FP8MLP_ERR_ARG;
+    if (c == nullptr || sc == nullptr) return FP8MLP_ERR_ARG;
+    const bool cast_done = mode == FP8MLP_SCALE_GIVEN_WEIGHTS_CAST;      // the FP8 weight buffers are already filled
+    if (!cast_done && (W1 == nullptr || W2 == nullptr || W3 == nullptr)) return FP8MLP_ERR_ARG;
+    if (mode != FP8MLP_SCALE_GIVEN && mode != FP8MLP_SCALE_FROM_CURRENT_AMAX && !cast_done) return FP8MLP_ERR_ARG;
+    if (cast_done && (c->flags & FP8MLP_H_BF16)) return FP8MLP_ERR_ARG;  // that variant keeps W3 in bf16, not as codes
     if (!on_device_of(c)) return FP8MLP_ERR_STATE;
     if (T < 0 || T > c->T_max) return FP8MLP_ERR_SHAPE;
     if (T > 0 && (x == nullptr || y == nullptr)) return FP8MLP_ERR_ARG;
@@ -276,6 +294,9 @@ int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_
                        (void**)&c->gu, (void**)&c->dyq, (void**)&c->dzq, (void**)&c->hb, (void**)&c->w3b};
     for (int i = 0; i < 9 && e == cudaSuccess; ++i) e = cudaMalloc(slots[i], static_cast<size_t>(c->bytes[i]));
     if (e == cudaSuccess) e = cudaMalloc((void**)&c->dummy, sizeof(float) * (8 + f));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&c->splitk_ws, sizeof(float) * kSplitFloats);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&c->splitk_cnt, sizeof(unsigned int) * kSplitWords);
+    if (e == cudaSuccess) e = cudaMemset(c->splitk_cnt, 0, sizeof(unsigned int) * kSplitWords);
     if (e == cudaSuccess) e = cudaMalloc((void**)&c->status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int));
     if (e != cudaSuccess) {
@@ -289,7 +310,7 @@ int fp8mlp_create(fp8mlp_ctx** out, int64_t T_max, int64_t d, int64_t f, uint32_
 
 int fp8mlp_destroy(fp8mlp_ctx* c) {
     if (c == nullptr) return FP8MLP_OK;
-    void* ptrs[] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq, c->hb, c->w3b, c->dummy, c->status};
+    void* ptrs[] = {c->xq, c->w12q, c->w3q, c->hq, c->gu, c->dyq, c->dzq, c->hb, c->w3b, c->dummy, c->status, c->splitk_ws, c->splitk_cnt};
     for (void* p : ptrs)
         if (p != nullptr) cudaFree(p);
     if (c->brackets != nullptr) {
@@ -374,7 +395,7 @@ int fp8mlp_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, 
     int dev = 0, sms = 0;
     FP8MLP_CUDA_CHECK(cudaGetDevice(&dev));
     FP8MLP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    if (amax != nullptr) FP8MLP_TRY(zero_floats({amax}, st));
+    if (amax != nullptr) FP8MLP_TRY(zero_floats(nullptr, {amax}, st));
     if (scale_mode == FP8MLP_SCALE_FROM_CURRENT_AMAX)
         return quantize_tensor(src, src_dtype, rows, cols, fp8_fmt, scale_mode, scale, amax, nullptr, row_mul, nullptr, dst,
                                ld_dst, sms, st);
@@ -404,6 +425,8 @@ int fp8mlp_update_scales(fp8mlp_ctx* c, const fp8mlp_amax* am, fp8mlp_scales* sc
 int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, const float* W2, const float* W3,
                    int mode, fp8mlp_scales* sc, fp8mlp_amax* am, void* y, void* stream) {
     FP8MLP_TRY(check_forward_args(c, T, x, W1, W2, W3, mode, sc, am, y));
+    const bool weights_cast = mode == FP8MLP_SCALE_GIVEN_WEIGHTS_CAST;
+    if (weights_cast) mode = FP8MLP_SCALE_GIVEN;
     const bool gu_fp8 = (c->flags & FP8MLP_GU_FP8) != 0;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool smooth = (c->flags & FP8MLP_SMOOTH) != 0;
@@ -420,7 +443,8 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
 
     {
         PhaseTimer pt(c, FP8MLP_PH_MISC, st);
-        FP8MLP_TRY(zero_floats({a_x, a_w1, a_w2, a_w3, a_gu}, st, a_h, f));
+        if (weights_cast) FP8MLP_TRY(zero_floats(c, {a_x, a_gu}, st, a_h, f));     // the weights' maxima came with their codes
+        else FP8MLP_TRY(zero_floats(c, {a_x, a_w1, a_w2, a_w3, a_gu}, st, a_h, f));
     }
     {   // x -> E4M3
         PhaseTimer pt(c, FP8MLP_PH_QUANT_X, st);
@@ -453,7 +477,9 @@ int fp8mlp_forward(fp8mlp_ctx* c, int64_t T, const void* x, const float* W1, con
         if (c->flags & FP8MLP_SAVE_FOR_BWD) c->saved_T = T;
         return FP8MLP_OK;
     }
-    if (mode == FP8MLP_SCALE_GIVEN) {
+    if (weights_cast) {
+        // nothing to do: the optimizer step wrote this step's [W2 | W1] and W3' codes (fp8mlp_adam_step_cast)
+    } else if (mode == FP8MLP_SCALE_GIVEN) {
         // every scale is known: [W2 | W1] (one scale) and W3' = diag(1/s) W3 in one pass over the masters;
         // the reciprocal of s_i is taken inside the pass, row by row
         PhaseTimer pt(c, FP8MLP_PH_QUANT_W12, st);
@@ -519,7 +545,7 @@ int fp8mlp_merge_weights(fp8mlp_ctx* c, const float* W1, const float* W2, const 
     float* a_w3 = (am && am->w3) ? am->w3 : c->dummy + 3;
     c->saved_T = -1;
     c->merged = false;
-    FP8MLP_TRY(zero_floats({a_w1, a_w2, a_w3}, st));
+    FP8MLP_TRY(zero_floats(c, {a_w1, a_w2, a_w3}, st));
     QuantTensor t[3] = {};
     t[0].src = W2; t[0].rows = d; t[0].cols = f; t[0].dst = c->w12q; t[0].ld_dst = 2 * f; t[0].amax = a_w2;
     t[1].src = W1; t[1].rows = d; t[1].cols = f; t[1].dst = c->w12q + f; t[1].ld_dst = 2 * f; t[1].amax = a_w1;
@@ -555,7 +581,7 @@ int fp8mlp_forward_merged(fp8mlp_ctx* c, int64_t T, const void* x, int mode, fp8
     if (T == 0) return FP8MLP_OK;
     {
         PhaseTimer pt(c, FP8MLP_PH_MISC, st);
-        FP8MLP_TRY(zero_floats({a_x}, st, a_h, f));
+        FP8MLP_TRY(zero_floats(c, {a_x}, st, a_h, f));
     }
     {
         PhaseTimer pt(c, FP8MLP_PH_QUANT_X, st);
@@ -606,7 +632,7 @@ int fp8mlp_backward(fp8mlp_ctx* c, int64_t T, const void* dy, int mode, fp8mlp_s
     float* a_dz = (am && am->dz) ? am->dz : c->dummy + 5;
     {
         PhaseTimer pt(c, FP8MLP_PH_MISC, st);
-        FP8MLP_TRY(zero_floats({a_dy, a_dz}, st));
+        FP8MLP_TRY(zero_floats(c, {a_dy, a_dz}, st));
     }
     if (T == 0) {   // empty batch: the weight gradients are sums over no tokens
         FP8MLP_CUDA_CHECK(cudaMemsetAsync(dW1, 0, sizeof(float) * d * f, st));
@@ -720,6 +746,7 @@ int fp8mlp_forward_static(int64_t T, int64_t d, int64_t f, uint32_t flags, const
                           const float* W2, const float* W3, int mode, fp8mlp_scales* sc, fp8mlp_amax* am, void* y,
                           void* stream) {
     if (flags & ~uint32_t(FP8MLP_SMOOTH)) return FP8MLP_ERR_ARG;
+    if (mode == FP8MLP_SCALE_GIVEN_WEIGHTS_CAST) return FP8MLP_ERR_ARG;      // nothing persists in the built-in scratch
     if (T < 0 || d <= 0 || f <= 0 || d % 16 != 0 || f % 16 != 0) return FP8MLP_ERR_SHAPE;
     if (T > (1 << 22) || d > (1 << 22) || f > (1 << 22)) return FP8MLP_ERR_TOO_LARGE;
     if (T * d + 3 * d * f + T * f + 8 * f + 4096 > int64_t(FP8MLP_STATIC_SCRATCH_BYTES)) return FP8MLP_ERR_TOO_LARGE;

@@ -31,6 +31,30 @@ void count_launch();
         FP8MLP_CUDA_CHECK(cudaGetLastError());                    \
     } while (0)
 
+// Launch of a kernel of this library with programmatic stream serialisation: the grid may be set up
+// (blocks scheduled, their prologues run) while its predecessor in the stream is still draining, which
+// hides the launch latency between the dozen kernels of a step.  Every kernel launched this way calls
+// grid_dependency_wait() before its first access to global memory; that call returns once the
+// predecessor grid has completed and its writes are visible, so the data flow is that of an ordinary
+// in-order stream.
+#ifdef __CUDACC__
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Device status word values (written by kernels that give up on a bounded wait).
 enum : int { STATUS_OK = 0, STATUS_WAIT_TIMEOUT = 1 };
 
@@ -45,6 +69,11 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+
+// Programmatic dependent launch (see launch_chained): wait for the predecessor grid and its memory;
+// then let the successor grid be set up behind this one.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ---------------------------------------------------------------- FP8 / bf16 conversions
 // Two floats -> two FP8 codes (lo in bits 0-7, hi in bits 8-15), round-to-nearest-even,
@@ -214,6 +243,23 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t smem_dst, const CUtens
         : "memory");
 }
 
+// 2-D tile store shared -> global (bulk async group of the issuing thread); rows / columns of the box that lie
+// outside the tensor are not written.  x = innermost coordinate (a multiple of 16 bytes), never negative.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t smem_src, int32_t x, int32_t y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all of this thread's bulk stores have read their shared-memory source / have completed
+template <int PENDING>      // ... except for the PENDING most recent groups
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(PENDING) : "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// makes this thread's shared-memory writes visible to the bulk-copy engine
+__device__ __forceinline__ void fence_smem_to_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 // ---------------------------------------------------------------- tcgen05 (5th-gen tensor cores, TMEM)
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t ncols) {   // whole warp
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");
@@ -370,6 +416,11 @@ __device__ __forceinline__ void ld_global_nc_v8(const void* p, uint32_t (&w)[8])
 }
 __device__ __forceinline__ void ld_global_v8(const void* p, uint32_t (&w)[8]) {     // data the kernel also writes
     asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p) : "memory");
+}
+__device__ __forceinline__ void ld_global_cg_v8(const void* p, uint32_t (&w)[8]) {  // data other SMs wrote during this kernel: L2 only
+    asm volatile("ld.global.cg.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                  : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
                  : "l"(p) : "memory");
 }

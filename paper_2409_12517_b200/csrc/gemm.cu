@@ -10,10 +10,14 @@ namespace {
 // ---------------------------------------------------------------- shared memory plan
 // Single CTA: a stage holds an A box and two B boxes (128 x 256 tile).  CTA pair: a stage holds this
 // CTA's A box and its one B box (its halves of a 256 x 256 tile).
-// The backward SwiGLU kernel gives up stages for a ring of two 32-KiB slots through which a loader
-// warp streams the saved G and U (a 128-row x 64-channel bf16 box each) to the epilogue.
-constexpr int kGuSlots = 2;
-constexpr int kGuSlotBytes = 2 * kBoxBytes;
+// The backward SwiGLU kernel gives up a stage for a ring of three 16-KiB slots through which a loader warp
+// streams the saved G and U to the epilogue: a slot holds a box of 128 rows x 64 bytes of G and one of U
+// (32 channels as bf16, consumed by the four warps of one column half; or 64 channels as E4M3 codes,
+// consumed by all eight), 64-byte swizzle.  The main loop is sensitive to its depth - with three operand stages this
+// kernel runs 14 % slower than with four - so the ring is kept as small as hides the latency of its own loads.
+constexpr int kGuSlots = 3;
+constexpr int kGuBoxBytes = 128 * 64;
+constexpr int kGuSlotBytes = 2 * kGuBoxBytes;
 // WIDEN (CTA pairs, plain epilogues): a 256 x 512 tile - both accumulators belong to one tile, the A block
 // of a stage is loaded once for two B blocks (a quarter less operand traffic), the epilogue is not overlapped.
 template <bool PAIR, int EPI, bool WIDEN> struct Plan;
@@ -21,11 +25,19 @@ template <int EPI, bool WIDEN> struct Plan<false, EPI, WIDEN> {
     static constexpr int kStages = EPI == EPI_SWIGLU_BWD ? 3 : 4, kStageBytes = 3 * kBoxBytes, kTileM = 128;
 };
 template <int EPI, bool WIDEN> struct Plan<true, EPI, WIDEN> {
-    static constexpr int kStages = (EPI == EPI_SWIGLU_BWD || WIDEN) ? 4 : 6, kStageBytes = (WIDEN ? 3 : 2) * kBoxBytes, kTileM = 256;
+    static constexpr int kStages = WIDEN ? 4 : EPI == EPI_SWIGLU_BWD ? 5 : 6, kStageBytes = (WIDEN ? 3 : 2) * kBoxBytes, kTileM = 256;
 };
 constexpr int kMaxStages = 6;
+// With a short contraction (few tokens) the fp32-output kernels (weight gradients) are bound by their output, and a
+// thread owns a row of the accumulator, so direct stores touch 32 different lines per instruction and cost several
+// times the data-pipe cycles.  Then the output is staged in shared memory, in 32-row x 32-column blocks (4 KiB,
+// 128-byte swizzle) per epilogue warp, and sent to global memory as bulk tensor stores.  The staging blocks take the
+// place of the last two operand stages, which a short contraction does not need (args.stages, args.tma_store).
+constexpr int kStoreBlockBytes = 32 * 128;
+constexpr int kStagesLentToStores = 2;
 
-struct __align__(8) SmemTail {
+template <bool FUSED>            // FUSED: the SwiGLU epilogues, which keep per-channel scales and maxima of the tile here
+struct __align__(8) SmemTailT {
     uint64_t full[kMaxStages];   // TMA -> MMA: stage filled (CTA pair: only rank 0's are used)
     uint64_t empty[kMaxStages];  // MMA -> TMA: stage drained
     uint64_t tmem_full[2];       // MMA -> epilogue: accumulator complete
@@ -34,14 +46,18 @@ struct __align__(8) SmemTail {
     uint64_t gu_empty[kGuSlots]; // epilogue -> loader: chunk read into registers
     uint32_t tmem_base;
     int abort;
-    float s_tile[2][kBlockN];    // per-channel scales of the current tile(s)
-    unsigned int amax_tile[128]; // per-channel maxima of the current tile (forward)
+    float s_tile[2][FUSED ? kBlockN : 1];    // per-channel scales of the current tile(s)
+    unsigned int amax_tile[FUSED ? 128 : 1]; // per-channel maxima of the current tile (forward)
 };
+using SmemTail = SmemTailT<true>;
+template <int EPI> using TailOf = SmemTailT<EPI == EPI_SWIGLU_FWD || EPI == EPI_SWIGLU_BWD>;
 template <bool PAIR, int EPI, bool WIDEN>
 constexpr size_t smem_bytes() {
     return 1024 /*alignment slack*/ + size_t(Plan<PAIR, EPI, WIDEN>::kStages) * Plan<PAIR, EPI, WIDEN>::kStageBytes +
-           (EPI == EPI_SWIGLU_BWD ? size_t(kGuSlots) * kGuSlotBytes : 0) + sizeof(SmemTail);
+           (EPI == EPI_SWIGLU_BWD ? size_t(kGuSlots) * kGuSlotBytes : 0) + sizeof(TailOf<EPI>);
 }
+static_assert(smem_bytes<true, EPI_F32, false>() <= 232448 && smem_bytes<false, EPI_F32, false>() <= 232448 &&
+              smem_bytes<true, EPI_SWIGLU_BWD, false>() <= 232448, "shared memory plan exceeds what a CTA can have");
 
 // ---------------------------------------------------------------- descriptors
 // Shared-memory matrix descriptor, 128-byte swizzle.  Bits: [0,14) address>>4, [16,30) leading
@@ -166,6 +182,49 @@ __device__ __forceinline__ void epilogue_f32(const GemmArgs& p, uint32_t taddr, 
     }
 }
 
+// The same through shared memory: the thread writes its row's 32 values into one of the warp's NBUF staging blocks
+// (16-byte piece j of row r at piece j ^ (r & 7): the 128-byte swizzle, so the writes are free of bank conflicts and
+// the block is what a swizzled tensor-map box expects), one lane sends the block off as a bulk tensor store.  Rows
+// past M and columns past the output's width are cut off by the tensor map.  A chunk that straddles the boundary
+// between the two outputs of a split output is stored directly.  `blocks_sent` counts the warp's blocks.
+template <int NBUF>
+__device__ __forceinline__ void epilogue_f32_staged(const GemmArgs& p, const CUtensorMap* out0, const CUtensorMap* out1,
+                                                    uint32_t warp_stage_addr, uint32_t& blocks_sent, uint32_t taddr, int lane,
+                                                    int half, int m, int row0, int n0, float dq) {
+    const bool row_ok = m < p.M;
+#pragma unroll 1
+    for (int jj = 0; jj < 4; ++jj) {
+        const int j = 4 * half + jj;
+        const int c0 = n0 + 32 * j;
+        if (c0 >= p.N) break;
+        uint32_t r[32];
+        tmem_ld32(taddr + 32 * j, r);
+        tmem_ld_wait();
+        float v[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) v[e] = __fmul_rn(__uint_as_float(r[e]), dq);
+        if (c0 < p.n_split && c0 + 32 > p.n_split) {       // straddles the two outputs
+            if (row_ok) store_f32x32(p, v, m, c0);
+            continue;
+        }
+        const uint32_t block = warp_stage_addr + (blocks_sent % NBUF) * kStoreBlockBytes;
+        ++blocks_sent;
+        if (lane == 0) tma_store_wait_read<NBUF - 1>();    // the store that used this block last has read it
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            st_shared_v4(block + static_cast<uint32_t>(lane) * 128u + static_cast<uint32_t>((q ^ (lane & 7)) * 16),
+                         __float_as_uint(v[4 * q]), __float_as_uint(v[4 * q + 1]), __float_as_uint(v[4 * q + 2]), __float_as_uint(v[4 * q + 3]));
+        fence_smem_to_async_proxy();
+        __syncwarp();
+        if (lane == 0) {
+            if (c0 < p.n_split) tma_store_2d(out0, block, c0, row0);
+            else tma_store_2d(out1, block, c0 - p.n_split, row0);
+            tma_store_commit();
+        }
+    }
+}
+
 // 16 floats -> 16 bf16 (32 bytes) at dst, columns guarded by the caller
 __device__ __forceinline__ void store_bf16x16(uint16_t* dst, const float* v, bool wide) {
     uint32_t w[8];
@@ -196,6 +255,79 @@ __device__ __forceinline__ void epilogue_bf16(const GemmArgs& p, uint32_t taddr,
         uint16_t* dst = p.out_bf16 + static_cast<int64_t>(m) * p.ld_out + c0;
         store_bf16x16(dst, v, p.wide);
         if (c0 + 16 < p.N) store_bf16x16(dst + 16, v + 16, p.wide);
+    }
+}
+
+// Split contraction: this CTA pair holds one of split_k partial sums of the tile.  The warp writes its raw fp32
+// partial (32 rows x 128 columns) to the workspace and counts itself; the warp that finds all the others of its
+// region already counted adds the split_k partials in split order - whichever warp that is, the sum is the same -
+// applies the dequantisation and writes the output.  Nothing waits: every warp but the last just leaves.
+template <int EPI>
+__device__ __forceinline__ void epilogue_split(const GemmArgs& p, uint32_t taddr, int lane, int half, unsigned int* counter,
+                                               int split, int m, int n0, float dq) {
+    const bool row_ok = m < p.M;
+    float* mine = p.partial + (static_cast<int64_t>(split) * p.M + m) * p.N;
+#pragma unroll 1
+    for (int jj = 0; jj < 4; ++jj) {
+        const int c0 = n0 + 32 * (4 * half + jj);
+        if (c0 >= p.N) break;
+        uint32_t r[32];
+        tmem_ld32(taddr + 32 * (4 * half + jj), r);
+        tmem_ld_wait();
+        if (!row_ok) continue;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (c0 + 8 * q >= p.N) break;
+            const uint32_t w[8] = {r[8 * q], r[8 * q + 1], r[8 * q + 2], r[8 * q + 3], r[8 * q + 4], r[8 * q + 5], r[8 * q + 6], r[8 * q + 7]};
+            st_global_v8(mine + c0 + 8 * q, w);
+        }
+    }
+    __threadfence();                       // this lane's partials are visible device-wide before the count
+    __syncwarp();
+    unsigned int before = 0;
+    if (lane == 0) before = atomicAdd(counter, 1u);
+    before = __shfl_sync(0xffffffffu, before, 0);
+    if (before != static_cast<unsigned int>(p.split_k - 1)) return;
+    __threadfence();                       // the other splits' partials, counted before ours, are visible now
+    if (lane == 0) *counter = 0u;          // every split has counted: ready for the next launch
+    if (!row_ok) return;
+#pragma unroll 1
+    for (int jj = 0; jj < 4; ++jj) {
+        const int c0 = n0 + 32 * (4 * half + jj);
+        if (c0 >= p.N) break;
+        float v[32] = {};
+        // two splits' rows are fetched at a time, so that their trips to L2 overlap; added in split order
+        for (int s = 0; s < p.split_k; s += 2) {
+            const bool two = s + 1 < p.split_k;
+            const float* first = p.partial + (static_cast<int64_t>(s) * p.M + m) * p.N + c0;
+            const float* second = first + static_cast<int64_t>(p.M) * p.N;
+            uint32_t w0[4][8], w1[4][8];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const bool in = c0 + 8 * q < p.N;
+                if (in) ld_global_cg_v8(first + 8 * q, w0[q]);
+                if (in && two) ld_global_cg_v8(second + 8 * q, w1[q]);
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (c0 + 8 * q >= p.N) break;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    float t = s == 0 ? __uint_as_float(w0[q][e]) : __fadd_rn(v[8 * q + e], __uint_as_float(w0[q][e]));
+                    if (two) t = __fadd_rn(t, __uint_as_float(w1[q][e]));
+                    v[8 * q + e] = t;
+                }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) v[e] = __fmul_rn(v[e], dq);
+        if constexpr (EPI == EPI_F32) {
+            store_f32x32(p, v, m, c0);
+        } else {
+            uint16_t* dst = p.out_bf16 + static_cast<int64_t>(m) * p.ld_out + c0;
+            store_bf16x16(dst, v, p.wide);
+            if (c0 + 16 < p.N) store_bf16x16(dst + 16, v + 16, p.wide);
+        }
     }
 }
 
@@ -292,16 +424,17 @@ __device__ __forceinline__ void epilogue_swiglu_fwd(const GemmArgs& p, SmemTail*
 }
 
 // Backward: accumulator = dY W3'^T for 256 channels, worked through in four chunks of 64 channels; of
-// each chunk this warp takes channels [32 half, 32 half + 32).  The saved bf16 G and U of a chunk arrive
-// in shared memory (loader warp, TMA, 128-byte swizzle: the 16-byte piece j of row r sits at piece
-// j ^ (r & 7)); the thread copies its row's 64 + 64 bytes to registers and hands the slot back.
-// Kept as E4M3 codes instead (p.gu8), a slot holds 128 channels of G and of U - two chunks - the thread
-// copies 32 + 32 bytes per chunk, hands the slot back after the second, and G = code * (1 / sgu).
+// each chunk this warp takes channels [32 half, 32 half + 32).  The saved bf16 G and U of those 32 channels
+// arrive in a ring slot of their own (loader warp, TMA, 64-byte swizzle: the 16-byte piece j of row r sits at
+// piece j ^ ((r >> 1) & 3)), read by the four warps of this column half; the thread copies its row's 64 + 64
+// bytes to registers and hands the slot back (the warps of the other half pass the slot without reading).  Kept as E4M3 codes instead (p.gu8), a slot holds all 64 channels
+// of the chunk, shared by all eight warps; the thread copies 32 + 32 bytes and G = code * (1 / sgu).
 // dH = acc * dq (* s_i with Smooth-SwiGLU); dU = dH * G sigma(G);
 // dG = dH * U * sigma(G) (1 + G (1 - sigma(G))); max of |dG|, |dU|; dZq = Q_e5m2([dG | dU] * sdz).
+// gu_fill: the ring fills this warp has passed (fills are numbered as the loader issues them).
 // Returns false if a wait ran out.  GU8: the saved activations are E4M3 codes (p.gu8), else bf16 (p.gu).
 template <bool GU8>
-__device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail* tail, uint32_t gu_base, uint32_t& gu_count,
+__device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail* tail, uint32_t gu_base, uint32_t& gu_fill,
                                                     const float* s_tile, uint32_t taddr, int lane, int half, int row,
                                                     int m, int n0, float dq, float sdz, float inv_sgu,
                                                     volatile int* abort_flag, float& run_max) {
@@ -316,39 +449,40 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
     if (fold) dq = __fmul_rn(dq, sdz);
 #pragma unroll 1
     for (int c = 0; c < 4; ++c) {
-        const uint32_t slot = gu_count % kGuSlots, phase = (gu_count / kGuSlots) & 1u;
         const int col = 64 * c + 32 * half;            // first of this warp's 32 accumulator columns
         const int c0 = n0 + col;
-        if (!gu8 || (c & 1) == 0) {                    // codes: the slot of chunk c - 1 also holds chunk c
+        uint4 gq[4], uq[4];
+        // Every warp passes every fill of the ring in order, whether the fill is for its column half or not: a
+        // barrier's parity only tells consecutive phases apart, so a warp that skipped a fill could take a slot's
+        // previous phase for the one it waits for (loads do not land in the order they were issued).
+#pragma unroll
+        for (int k = 0; k < (gu8 ? 1 : 2); ++k) {
+            const uint32_t slot = gu_fill % kGuSlots, phase = (gu_fill / kGuSlots) & 1u;
             // the warp leaves together or not at all: a wait that ran out for some lanes only would split it
             // between the failure path and the warp-wide instructions below
             const bool landed = mbar_wait(smem_u32(&tail->gu_full[slot]), phase, abort_flag, p.status);
             if (!__all_sync(0xffffffffu, landed)) return false;
-        }
-        uint4 gq[4], uq[4];
-        {
-            const uint32_t rbase = gu_base + slot * kGuSlotBytes + static_cast<uint32_t>(row) * 128u;
+            const uint32_t rbase = gu_base + slot * kGuSlotBytes + static_cast<uint32_t>(row) * 64u;
+            const uint32_t sw = static_cast<uint32_t>((row >> 1) & 3);
             if constexpr (gu8) {
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
-                    const uint32_t off = static_cast<uint32_t>(((4 * (c & 1) + 2 * half + i) ^ (row & 7)) * 16);
+                    const uint32_t off = ((static_cast<uint32_t>(2 * half + i)) ^ sw) * 16u;
                     gq[i] = ld_shared_v4(rbase + off);
-                    uq[i] = ld_shared_v4(rbase + kBoxBytes + off);
+                    uq[i] = ld_shared_v4(rbase + kGuBoxBytes + off);
                 }
                 gq[2] = gq[3] = uq[2] = uq[3] = make_uint4(0u, 0u, 0u, 0u);
-            } else {
+            } else if (k == half) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const uint32_t off = static_cast<uint32_t>(((4 * half + i) ^ (row & 7)) * 16);
+                    const uint32_t off = (static_cast<uint32_t>(i) ^ sw) * 16u;
                     gq[i] = ld_shared_v4(rbase + off);
-                    uq[i] = ld_shared_v4(rbase + kBoxBytes + off);
+                    uq[i] = ld_shared_v4(rbase + kGuBoxBytes + off);
                 }
             }
-        }
-        __syncwarp();
-        if (!gu8 || (c & 1) == 1) {
-            if (lane == 0) mbar_arrive(smem_u32(&tail->gu_empty[slot]));     // the slot's data is in registers
-            ++gu_count;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tail->gu_empty[slot]));     // this warp is done with the slot
+            ++gu_fill;
         }
         if (c0 >= f) continue;
         uint32_t acc[32];
@@ -441,11 +575,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     uint8_t* tiles_ptr = smem_raw + (tiles_addr - raw_addr);
     constexpr uint32_t kRingBytes = EPI == EPI_SWIGLU_BWD ? kGuSlots * kGuSlotBytes : 0;
     const uint32_t gu_base = tiles_addr + kStages * kStageBytes;     // ring of saved G, U chunks (backward only)
-    SmemTail* tail = reinterpret_cast<SmemTail*>(tiles_ptr + size_t(kStages) * kStageBytes + kRingBytes);
+    const uint32_t store_base = tiles_addr + static_cast<uint32_t>(p.stages) * kStageBytes;   // staging blocks of the fp32 output, if used
+    using Tail = TailOf<EPI>;
+    Tail* tail = reinterpret_cast<Tail*>(tiles_ptr + size_t(kStages) * kStageBytes + kRingBytes);
+    const uint32_t n_stages = static_cast<uint32_t>(p.stages);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int num_tiles = p.num_m_tiles * p.num_n_tiles;
+    // a work item is a tile, or with a split contraction one of a tile's split_k shares (shares of a tile are
+    // neighbouring items, so they run at the same time on neighbouring CTA pairs)
+    const int num_tiles = p.num_m_tiles * p.num_n_tiles * p.split_k;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;             // rank in the CTA pair
     const int first_tile = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
     const int tile_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
@@ -478,6 +617,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if constexpr (PAIR) cluster_sync_all(); else __syncthreads();   // barriers of both CTAs are ready
     tc_fence_after();
     const uint32_t tmem_base = tail->tmem_base;
+    // Everything above touched only this CTA's shared and tensor memory and may have run while the previous
+    // kernel of the stream was still finishing; from here on its results are needed.
+    grid_dependency_wait();
+    grid_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -486,13 +629,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             bool ok = true;
             const CUtensorMap* tmB = (PAIR && rank != 0) ? &tmB1 : &tmB0;
             const uint64_t pol_a = l2_policy(p.hint_a), pol_b = l2_policy(p.hint_b);
-            for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step) {
+            for (int item = first_tile; ok && item < num_tiles; item += tile_step) {
                 int m_tile, n_tile;
+                const int tile = item / p.split_k, split = item - tile * p.split_k;
                 tile_coords(p, tile, m_tile, n_tile);
                 const int m0 = m_tile * kTileM + static_cast<int>(rank) * kBlockM;
                 const int nb0 = n_tile * p.n_tile_cols + (PAIR ? static_cast<int>(rank) * p.b1_offset : 0);
                 const int nb1 = nb0 + p.b1_offset;
-                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                const int kb_end = min(p.num_k_blocks, (split + 1) * p.kb_per_split);
+                for (int kb = split * p.kb_per_split; kb < kb_end; ++kb) {
                     if (!mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     const uint32_t dst = tiles_addr + stage * kStageBytes;
                     const int k0 = kb * (kBlockK / ELEM);          // in elements
@@ -510,7 +655,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         load_operand<B_MN, ELEM, false>(dst + kBoxBytes, &tmB0, bar, nb0, k0, p.hint_b, pol_b);
                         load_operand<B_MN, ELEM, false>(dst + 2 * kBoxBytes, &tmB1, bar, nb1, k0, p.hint_b, pol_b);
                     }
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
                 }
             }
         }
@@ -520,12 +665,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             int it = 0;
-            for (int tile = first_tile; ok && tile < num_tiles; tile += tile_step, ++it) {
+            for (int item = first_tile; ok && item < num_tiles; item += tile_step, ++it) {
                 const uint32_t acc = WIDEN ? 0u : (it & 1), acc_phase = WIDEN ? (it & 1) : ((it >> 1) & 1);
                 if (!mbar_wait(smem_u32(&tail->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, p.status)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kBlockN;
-                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                const int split = item % p.split_k;
+                const int kb_begin = split * p.kb_per_split, kb_end = min(p.num_k_blocks, kb_begin + p.kb_per_split);
+                for (int kb = kb_begin; kb < kb_end; ++kb) {
                     if (!mbar_wait(smem_u32(&tail->full[stage]), phase, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = tiles_addr + stage * kStageBytes;
@@ -534,7 +681,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                         const uint64_t da = smem_desc<A_MN, ELEM>(a_addr + k * k_step_bytes<A_MN, ELEM>());
                         const uint64_t db = smem_desc<B_MN, ELEM>(b_addr + k * k_step_bytes<B_MN, ELEM>());
-                        const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
+                        const uint32_t accum = (kb != kb_begin || k != 0) ? 1u : 0u;
                         if constexpr (WIDEN) {       // second half of the 512 columns: same A, the stage's other B block
                             const uint64_t db1 = smem_desc<B_MN, ELEM>(b_addr + kBoxBytes + k * k_step_bytes<B_MN, ELEM>());
                             umma_f8_pair(d_tmem, da, db, p.idesc, accum);
@@ -548,7 +695,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     // frees the stage (in both CTAs) once these MMAs have read it
                     if constexpr (PAIR) umma_commit_pair(smem_u32(&tail->empty[stage]));
                     else umma_commit(smem_u32(&tail->empty[stage]));
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
                 }
                 if (ok) {
                     if constexpr (PAIR) umma_commit_pair(smem_u32(&tail->tmem_full[acc]));
@@ -569,16 +716,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     tile_coords(p, tile, m_tile, n_tile);
                     const int m0 = m_tile * kTileM + static_cast<int>(rank) * kBlockM;
                     const int n0 = n_tile * p.n_tile_cols;
-                    // per slot 64 channels of bf16 G and U, or 128 channels of their E4M3 codes: 4 or 2 slots a tile
-                    constexpr int n_slots = GU8 ? 2 : 4, per_slot = GU8 ? 128 : 64;
-                    for (int c = 0; c < n_slots; ++c, ++count) {
+                    // per fill 64 bytes of every row of G and of U: 32 channels as bf16 (8 fills a tile, alternating
+                    // between the two column halves of a 64-channel chunk) or 64 channels as E4M3 codes (4 fills)
+                    constexpr int n_fills = GU8 ? 4 : 8, per_fill = GU8 ? 64 : 32;
+                    for (int c = 0; c < n_fills; ++c, ++count) {
                         const uint32_t slot = count % kGuSlots, phase = (count / kGuSlots) & 1u;
                         if (!mbar_wait(smem_u32(&tail->gu_empty[slot]), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
                         const uint32_t bar = smem_u32(&tail->gu_full[slot]);
                         const uint32_t dst = gu_base + slot * kGuSlotBytes;
                         mbar_expect_tx(bar, kGuSlotBytes);
-                        tma_load_2d(dst, &tmG, bar, n0 + per_slot * c, m0);        // columns past f read as zeros
-                        tma_load_2d(dst + kBoxBytes, &tmU, bar, n0 + per_slot * c, m0);
+                        tma_load_2d(dst, &tmG, bar, n0 + per_fill * c, m0);        // columns past f read as zeros
+                        tma_load_2d(dst + kGuBoxBytes, &tmU, bar, n0 + per_fill * c, m0);
                     }
                 }
             }
@@ -597,10 +745,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if constexpr (EPI == EPI_SWIGLU_FWD || EPI == EPI_SWIGLU_BWD) {
             if constexpr (GU8) { sgu = *p.s_gu; inv_sgu = __fdiv_rn(1.0f, sgu); }
         }
-        uint32_t gu_count = 0;                         // chunks of saved G, U consumed so far (backward)
+        // staging blocks per warp for the fp32 output: what two lent stages hold, shared by the eight epilogue warps
+        constexpr int kStoreBlocks = (kStagesLentToStores * kStageBytes) / ((kEpiThreads / 32) * kStoreBlockBytes) >= 2 ? 2 : 1;
+        uint32_t blocks_sent = 0;
+        uint32_t gu_fill = 0;                          // ring fills of saved G, U this warp has passed (backward)
         int it = 0;
-        for (int tile = first_tile; tile < num_tiles; tile += tile_step, ++it) {
+        for (int item = first_tile; item < num_tiles; item += tile_step, ++it) {
             int m_tile, n_tile;
+            const int tile = item / p.split_k, split = item - tile * p.split_k;
             tile_coords(p, tile, m_tile, n_tile);
             const int m = m_tile * kTileM + static_cast<int>(rank) * kBlockM + row;
             const int n0 = n_tile * p.n_tile_cols;
@@ -620,15 +772,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 float dq = dq0;
                 if (p.row_s != nullptr)
                     dq = __fmul_rn(inv_or_one(p.s0), m < p.M ? __fdiv_rn(1.0f, p.row_s[m]) : 1.0f);
-                epilogue_f32(p, taddr, half, m, n0, dq);
+                if (!WIDEN && p.split_k > 1)
+                    epilogue_split<EPI_F32>(p, taddr, lane, half, p.tile_counters + tile * 16 + rank * 8 + (warp - 2), split, m, n0, dq);
+                else if (!WIDEN && p.tma_store)
+                    epilogue_f32_staged<kStoreBlocks>(p, &tmG, &tmU, store_base + static_cast<uint32_t>(warp - 2) * (kStoreBlocks * kStoreBlockBytes),
+                                                      blocks_sent, taddr, lane, half, m, m - lane, n0, dq);
+                else epilogue_f32(p, taddr, half, m, n0, dq);
                 if constexpr (WIDEN) epilogue_f32(p, taddr + kBlockN, half, m, n0 + kBlockN, dq);
             } else if constexpr (EPI == EPI_BF16) {
-                epilogue_bf16(p, taddr, half, m, n0, dq0);
+                if (!WIDEN && p.split_k > 1)
+                    epilogue_split<EPI_BF16>(p, taddr, lane, half, p.tile_counters + tile * 16 + rank * 8 + (warp - 2), split, m, n0, dq0);
+                else epilogue_bf16(p, taddr, half, m, n0, dq0);
                 if constexpr (WIDEN) epilogue_bf16(p, taddr + kBlockN, half, m, n0 + kBlockN, dq0);
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
                 epilogue_swiglu_fwd<GU8>(p, tail, taddr, lane, half, m, n0, dq0, sgu, gu_max);
             } else {
-                const bool fine = epilogue_swiglu_bwd<GU8>(p, tail, gu_base, gu_count, tail->s_tile[acc], taddr, lane, half, row,
+                const bool fine = epilogue_swiglu_bwd<GU8>(p, tail, gu_base, gu_fill, tail->s_tile[acc], taddr, lane, half, row,
                                                            m, n0, dq0, sdz, inv_sgu, abort_flag, run_max);
                 if (!epi_all(fine)) break;
             }
@@ -648,6 +807,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 // each thread resets only its own amax_tile / s_tile entry for the next tile, and the
                 // others touch them again only after the next tile's barrier: no second barrier needed
             }
+        }
+        if constexpr (EPI == EPI_F32) {
+            if (lane == 0) tma_store_wait_all();       // the staged output has reached global memory
         }
         if constexpr (EPI == EPI_SWIGLU_BWD) {
             run_max = warp_max_nonneg(run_max);
@@ -695,22 +857,35 @@ EncodeTiledFn encode_fn() {
 }
 
 template <int EPI, bool A_MN, bool B_MN, bool PAIR, int ELEM, bool WIDEN = false, bool GU8 = false>
-int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorMap& tmB1, const GemmArgs& args,
+int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorMap& tmB1, const GemmArgs& args_in,
                 int64_t tiles, int sm_count, cudaStream_t st) {
     constexpr size_t kSmem = smem_bytes<PAIR, EPI, WIDEN>();
+    GemmArgs args = args_in;
+    if (EPI != EPI_F32 || WIDEN) args.tma_store = 0;
+    args.stages = Plan<PAIR, EPI, WIDEN>::kStages - (args.tma_store ? kStagesLentToStores : 0);
     // the saved activations [M, 2f] bf16 as two matrices of f columns: G, and U starting f elements in
     CUtensorMap tmG = tmA, tmU = tmA;
     if constexpr (EPI == EPI_SWIGLU_BWD) {
         const uint64_t f = static_cast<uint64_t>(args.N), rows = static_cast<uint64_t>(args.M);
         int rc;
-        if (GU8) {                       // E4M3 codes [M, 2f]: boxes of 128 channels
-            rc = make_tmap_u8(&tmG, args.gu8, f, rows, 2 * f);
-            if (rc == FP8MLP_OK) rc = make_tmap_u8(&tmU, args.gu8 + f, f, rows, 2 * f);
-        } else {
-            rc = make_tmap(&tmG, args.gu, 2, false, f, rows, 4 * f);
-            if (rc == FP8MLP_OK) rc = make_tmap(&tmU, args.gu + f, 2, false, f, rows, 4 * f);
+        if (GU8) {                       // E4M3 codes [M, 2f]: boxes of 64 channels x 128 rows
+            rc = make_tmap_ring(&tmG, args.gu8, 1, f, rows, 2 * f);
+            if (rc == FP8MLP_OK) rc = make_tmap_ring(&tmU, args.gu8 + f, 1, f, rows, 2 * f);
+        } else {                         // bf16 [M, 2f]: boxes of 32 channels x 128 rows
+            rc = make_tmap_ring(&tmG, args.gu, 2, f, rows, 4 * f);
+            if (rc == FP8MLP_OK) rc = make_tmap_ring(&tmU, args.gu + f, 2, f, rows, 4 * f);
         }
         if (rc != FP8MLP_OK) return rc;
+    }
+    if constexpr (EPI == EPI_F32 && !WIDEN) {
+        if (args.tma_store) {                // the two outputs of a (possibly split) fp32 result, boxes of 32 x 32
+            const uint64_t rows = static_cast<uint64_t>(args.M), w0 = static_cast<uint64_t>(args.n_split < args.N ? args.n_split : args.N);
+            int rc = make_tmap_out_f32(&tmG, args.out_f32_0, w0, rows, static_cast<uint64_t>(args.ld_out) * 4);
+            if (rc == FP8MLP_OK && args.N > args.n_split)
+                rc = make_tmap_out_f32(&tmU, args.out_f32_1, static_cast<uint64_t>(args.N - args.n_split), rows,
+                                       static_cast<uint64_t>(args.ld_out) * 4);
+            if (rc != FP8MLP_OK) return rc;
+        }
     }
     // the function attribute and the occupancy answer belong to a device: looked up once per device
     constexpr int kMaxDevices = 64;
@@ -724,17 +899,21 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
     cudaError_t& attr_err = attr_err_dev[dev];
     int& max_clusters = max_clusters_dev[dev];
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     cfg.blockDim = dim3(kGemmThreads);
     cfg.dynamicSmemBytes = kSmem;
     cfg.stream = st;
+    // set up behind the previous kernel of the stream (see launch_chained); the kernel waits for it itself
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (PAIR) {
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = 2;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
     }
     std::call_once(once, [&] {
         attr_err = cudaFuncSetAttribute(gemm_kernel<EPI, A_MN, B_MN, PAIR, ELEM, WIDEN, GU8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -783,6 +962,40 @@ int make_tmap(CUtensorMap* map, const void* base, int elem_bytes, bool mn_major,
     return FP8MLP_OK;
 }
 
+int make_tmap_ring(CUtensorMap* map, const void* base, int elem_bytes, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return FP8MLP_ERR_CUDA;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {row_stride_bytes};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(64 / elem_bytes), 128};
+    const cuuint32_t elem[2] = {1, 1};
+    CUresult r = fn(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                    const_cast<void*>(base), dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_cuda_error_str("cuTensorMapEncodeTiled", "driver rejected the tensor map of the saved activations");
+        return FP8MLP_ERR_CUDA;
+    }
+    return FP8MLP_OK;
+}
+
+int make_tmap_out_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return FP8MLP_ERR_CUDA;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {row_stride_bytes};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t elem[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, elem,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_cuda_error_str("cuTensorMapEncodeTiled", "driver rejected the output tensor map");
+        return FP8MLP_ERR_CUDA;
+    }
+    return FP8MLP_OK;
+}
+
 int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride) {
     return make_tmap(map, base, 1, false, inner, outer, row_stride);
 }
@@ -805,7 +1018,24 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     const int elem = args.elem_bytes == 2 ? 2 : 1;
     const int kblk = kBlockK / elem;     // contraction elements per stage
     args.num_k_blocks = (args.K + kblk - 1) / kblk;
-    if (args.group <= 0) args.group = pair ? 8 : 16;
+    if (args.group <= 0) {
+        // Rasterisation.  A wave of tiles (one per CTA or CTA pair) streams a block of A rows and a block of B rows
+        // through L2 for the whole contraction; what the next wave can still find there is the slice of one operand
+        // that its tiles share with this wave's.  The plain GEMMs band along the smaller operand and cut it into
+        // as few bands as keep a band's slice near a third of L2 (measured at the 7B shapes: a quarter less DRAM
+        // reading than full-height bands, 1.6 % off the step); the fused-epilogue GEMMs read less with bands of 16
+        // row tiles.
+        args.group = 16;
+        args.band_n = 0;
+        if (epi == EPI_F32 || epi == EPI_BF16) {
+            const int64_t a_bytes = static_cast<int64_t>(args.M) * args.K * elem, b_bytes = static_cast<int64_t>(args.N) * args.K * elem;
+            constexpr int64_t kBandBytes = int64_t(46) << 20;
+            args.band_n = b_bytes < a_bytes ? 1 : 0;
+            const int64_t bands = ((args.band_n ? b_bytes : a_bytes) + kBandBytes - 1) / kBandBytes;
+            const int along = args.band_n ? args.num_n_tiles : args.num_m_tiles;
+            args.group = static_cast<int>((along + bands - 1) / bands);
+        }
+    }
     // instruction descriptor: [4,6) D = fp32; [7,10) A format; [10,13) B format (0 = E4M3, 1 = E5M2);
     // bit 15 / 16: A / B is MN-major; [17,23) N >> 3; [24,29) M >> 4 (M counts both CTAs of a pair)
     args.idesc = (1u << 4) | (static_cast<uint32_t>(a_fmt) << 7) | (static_cast<uint32_t>(b_fmt) << 10) |
@@ -819,8 +1049,28 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
         case EPI_SWIGLU_FWD: args.wide = al32(args.hq) && al32(args.gu8) && args.N % 32 == 0; break;
         default: args.wide = al32(args.dzq) && args.N % 32 == 0; break;
     }
-    const int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
+    // fp32 outputs leave as bulk tensor stores when every box is at least as wide as the output is (32 columns)
+    // (and when the contraction is so short that the kernel is bound by its output: at 16 stages' worth of work and
+    // beyond, direct stores hide behind the main loop and the staging only costs shared-memory bandwidth)
+    args.tma_store = (epi == EPI_F32 && !widen && args.num_k_blocks <= 8 && args.N >= 32 &&
+                      (args.n_split >= args.N || (args.n_split >= 32 && args.N - args.n_split >= 32))) ? 1 : 0;
+    int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
     if (tiles == 0 || args.num_k_blocks == 0) return FP8MLP_OK;
+    // A problem with fewer tiles than CTA pairs leaves SMs idle through a long contraction: split it.
+    args.split_k = 1;
+    args.kb_per_split = args.num_k_blocks;
+    if (pair && !widen && (epi == EPI_F32 || epi == EPI_BF16) && args.partial != nullptr && args.tile_counters != nullptr) {
+        const int64_t pairs = sm_count / 2;
+        int64_t want = pairs / tiles;                                   // shares per tile that still fit one wave
+        if (want > 8) want = 8;
+        while (want > 1 && args.num_k_blocks / want < 8) --want;        // a share keeps at least 8 stages' worth of work
+        while (want > 1 && want * static_cast<int64_t>(args.M) * args.N > args.partial_floats) --want;
+        if (want > 1 && tiles * 16 <= args.counter_words) {
+            args.kb_per_split = static_cast<int>((args.num_k_blocks + want - 1) / want);
+            args.split_k = (args.num_k_blocks + args.kb_per_split - 1) / args.kb_per_split;   // every share non-empty
+            tiles *= args.split_k;
+        }
+    }
 
 #define FP8MLP_DISPATCH_WIDE(E, AM, BM)                                                                     \
     if (widen && epi == E && a_mn == AM && b_mn == BM)                                                      \

@@ -42,7 +42,7 @@ struct GemmArgs {
     int num_m_tiles, num_n_tiles, num_k_blocks;
     int n_tile_cols;        // n coordinates per tile: 256, or 128 when the two B boxes are gate and linear halves
     int b1_offset;          // n offset of the second B box: 128, or 0 in the gate/linear case
-    int group;              // tiles per rasterisation band, counted along m (band_n = 0) or along n (band_n = 1)
+    int group;              // tiles per rasterisation band, counted along m (band_n = 0) or along n (band_n = 1); 0: chosen by the launcher
     int band_n;
     int hint_a, hint_b;     // L2 eviction priority of the A / B operand loads (L2_HINT_*)
     int pair_mode;          // 0: CTA pairs when M > 128; 1: always CTA pairs; 2: always single CTAs
@@ -50,6 +50,16 @@ struct GemmArgs {
     int wide_tiles;         // 256 x 512 tiles: 0 = for bf16 outputs (default), 1 = for fp32 outputs too, 2 = never
     uint32_t idesc;
     int* status;
+    // Split of the contraction over several CTA pairs (problems with fewer tiles than the GPU has CTA pairs;
+    // plain epilogues only).  Every split writes its fp32 partial tile to `partial` ([split_k][M][N]) and counts
+    // itself in tile_counters (16 words per tile: one per epilogue warp of the pair); the warp that arrives last
+    // for its 32 x 128 region adds the partials in split order and writes the output.  split_k = 1: off.
+    int split_k;
+    int kb_per_split;
+    float* partial;                 // workspace, nullable (then no split is made)
+    int64_t partial_floats;         // its capacity
+    unsigned int* tile_counters;    // zero before the launch; left zero by it
+    int counter_words;
 
     // dequantisation: dq = (1 / *s0) * (1 / *s1); a null pointer stands for 1
     const float* s0;
@@ -61,6 +71,9 @@ struct GemmArgs {
     float* out_f32_1;
     int n_split;
     int64_t ld_out;
+    int tma_store;          // set by the launcher: the fp32 output leaves through shared memory and bulk tensor stores
+    int stages;             // set by the launcher: operand stages in use (all of the kernel's, or two fewer when their
+                            // shared memory stages the output)
     // EPI_BF16: out_bf16[m*ld_out + n] = bf16(acc * dq)
     uint16_t* out_bf16;
     // SwiGLU epilogues (f = N)
@@ -89,6 +102,11 @@ int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t ou
 // the GEMM will read the matrix (an MN-major 16-bit operand is fetched in boxes of 64 K-rows).
 int make_tmap(CUtensorMap* map, const void* base, int elem_bytes, bool mn_major, uint64_t inner, uint64_t outer,
               uint64_t row_stride_bytes);
+
+// Tensor map of the saved activations for the backward epilogue's ring: boxes of 64 bytes x 128 rows, 64-byte swizzle.
+int make_tmap_ring(CUtensorMap* map, const void* base, int elem_bytes, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes);
+// Tensor map of an fp32 output matrix for bulk stores: boxes of 32 columns x 32 rows, 128-byte swizzle.
+int make_tmap_out_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes);
 
 // Launches one GEMM.  a_mn / b_mn: the operand is MN-major.  The tensor maps describe A, and the
 // two 128-wide halves of the B tile (the same map twice unless they come from different matrices).

@@ -90,6 +90,8 @@ template <typename SRC, int FMT, bool CAST, bool AMAX>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSm)
 quantize_kernel(const QuantLaunch q) {
     constexpr int E = Unit<SRC>::kElems;
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int seg_id = blockIdx.x % q.nseg;
     const QuantSeg& sg = q.seg[seg_id];
     const SRC* __restrict__ src = static_cast<const SRC*>(sg.src);
@@ -164,6 +166,8 @@ quantize_kernel(const QuantLaunch q) {
 
 // scale = fmt_max / max(amax_a, amax_b)   (amax_b nullable)
 __global__ void scale_kernel(int fmt, const float* amax_a, const float* amax_b, float* scale) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     float a = *amax_a;
     if (amax_b != nullptr) a = fmaxf(a, *amax_b);
     *scale = scale_from_amax_dev(fmt, a);
@@ -171,6 +175,8 @@ __global__ void scale_kernel(int fmt, const float* amax_a, const float* amax_b, 
 
 // One launch for the whole amax -> scale bookkeeping (see UpdateScalesArgs).
 __global__ void __launch_bounds__(kThreads) update_scales_kernel(UpdateScalesArgs a) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         if (a.amax_x && a.scale_x) *a.scale_x = scale_from_amax_dev(FP8MLP_E4M3, *a.amax_x);
         if (a.amax_w1 && a.amax_w2 && a.scale_w12)
@@ -210,6 +216,8 @@ __global__ void __launch_bounds__(kThreads) update_scales_kernel(UpdateScalesArg
 // fp32 -> bf16 (round to nearest even) with max |v|: the weight of a layer that is not quantised
 __global__ void __launch_bounds__(kThreads) cast_bf16_kernel(const float* __restrict__ src, uint16_t* __restrict__ dst,
                                                              int64_t n_units, float* amax_out) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     float local_max = 0.0f;
     for (int64_t u = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; u < n_units;
          u += static_cast<int64_t>(gridDim.x) * kThreads) {
@@ -225,9 +233,11 @@ __global__ void __launch_bounds__(kThreads) cast_bf16_kernel(const float* __rest
 
 template <typename SRC, int FMT>
 int launch_pass(bool cast, bool amax, const QuantLaunch& q, int grid, cudaStream_t st) {
-    if (cast && amax) quantize_kernel<SRC, FMT, true, true><<<grid, kThreads, 0, st>>>(q);
-    else if (cast) quantize_kernel<SRC, FMT, true, false><<<grid, kThreads, 0, st>>>(q);
-    else quantize_kernel<SRC, FMT, false, true><<<grid, kThreads, 0, st>>>(q);
+    cudaError_t e;
+    if (cast && amax) e = launch_chained(quantize_kernel<SRC, FMT, true, true>, grid, kThreads, 0, st, q);
+    else if (cast) e = launch_chained(quantize_kernel<SRC, FMT, true, false>, grid, kThreads, 0, st, q);
+    else e = launch_chained(quantize_kernel<SRC, FMT, false, true>, grid, kThreads, 0, st, q);
+    FP8MLP_CUDA_CHECK(e);
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
 }
@@ -306,13 +316,13 @@ int run_cast_bf16(const float* src, uint16_t* dst, int64_t n, float* amax_out, i
     if (units == 0) return FP8MLP_OK;
     int64_t blocks = (units + kThreads - 1) / kThreads;
     if (blocks > int64_t(sm_count) * 8) blocks = int64_t(sm_count) * 8;
-    cast_bf16_kernel<<<static_cast<int>(blocks), kThreads, 0, st>>>(src, dst, units, amax_out);
+    FP8MLP_CUDA_CHECK(launch_chained(cast_bf16_kernel, static_cast<int>(blocks), kThreads, 0, st, src, dst, units, amax_out));
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
 }
 
 int run_scale_from_amax(int fmt, const float* amax_a, const float* amax_b, float* scale, cudaStream_t st) {
-    scale_kernel<<<1, 1, 0, st>>>(fmt, amax_a, amax_b, scale);
+    FP8MLP_CUDA_CHECK(launch_chained(scale_kernel, 1, 1, 0, st, fmt, amax_a, amax_b, scale));
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
 }
@@ -321,7 +331,7 @@ int run_update_scales(const UpdateScalesArgs& a, int sm_count, cudaStream_t st) 
     int64_t blocks = a.amax_h ? (a.f + kThreads - 1) / kThreads : 1;
     if (blocks < 1) blocks = 1;
     if (blocks > sm_count) blocks = sm_count;
-    update_scales_kernel<<<static_cast<int>(blocks), kThreads, 0, st>>>(a);
+    FP8MLP_CUDA_CHECK(launch_chained(update_scales_kernel, static_cast<int>(blocks), kThreads, 0, st, a));
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
 }

@@ -135,3 +135,9 @@ PARITY_FIGURES = []
 
 def record_parity(test: str, **figures):
     PARITY_FIGURES.append(dict(test=test, **{k: (float(v) if isinstance(v, (np.floating, float)) else v) for k, v in figures.items()}))
+
+
+def code_diff(fmt, got_codes, ref_codes):
+    """dec(got) - dec(ref) in fp64: zero wherever the two sides stored the same code."""
+    import oracle
+    return oracle.decode(fmt, got_codes).astype(np.float64) - oracle.decode(fmt, ref_codes).astype(np.float64)

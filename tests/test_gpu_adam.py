@@ -132,3 +132,68 @@ def test_adam_argument_errors():
     assert L.fp8mlp_adam_step(arr, 1, 1e-3, 0.9, 0.95, 1e-8, 0.0, 0, None) == B.ERR_ARG      # step 0
     assert L.fp8mlp_adam_step(arr, 9, 1e-3, 0.9, 0.95, 1e-8, 0.0, 1, None) == B.ERR_ARG
     assert L.fp8mlp_launch_count() == n0
+
+
+def test_adam_step_that_also_casts_the_weights_for_the_next_forward():
+    """fp8mlp_adam_step_cast on the three weight matrices of a block, the codes going straight into a context's FP8
+    weight buffers ([W2 | W1] with one scale, W3' = diag(1/s) W3 with its own), then a forward that takes them as
+    they are.  Against the oracle (step, then its quantise routine): moments and their maxima bit for bit as in
+    the plain step; the weight codes equal except where the kernel's approximate square root and division moved a
+    weight across a rounding boundary (at most one step on at most 1e-4 of the codes), their maxima to 1e-6.
+    Against the CUDA path itself: the codes equal, bit for bit, what the forward's own weight pass makes of the
+    updated master weights, and the two forwards give the same output bit for bit."""
+    from helpers import bf16_dev_to_bits, code_mismatch
+    w = wl.make("ac", 17, 96, 128, 208, w_std=0.05, channel_outlier_frac=0.02)
+    T, d, f = w.T, w.d, w.f
+    rng = np.random.default_rng(5)
+    grads = [rng.normal(0, 1e-3, a.shape).astype(np.float32) for a in (w.W1, w.W2, w.W3)]
+    s_h = (2.0 ** rng.integers(-3, 5, f)).astype(np.float32)
+    sw12, sw3 = np.float32(2000.0), np.float32(700.0)
+    hp = dict(lr=1e-2, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.01)
+    ctx = B.fp8mlp_create(T, d, f, B.SMOOTH)
+    try:
+        sc, am = B.new_scales(f), B.new_amax(f)
+        sc["h"].copy_(to_dev(s_h)); sc["w12"].fill_(float(sw12)); sc["w3"].fill_(float(sw3)); sc["x"].fill_(64.0)
+        dev = [_dev_state(a) for a in (w.W1, w.W2, w.W3)]
+        for st, g in zip(dev, grads):
+            st["g"] = to_dev(g.ravel())
+        p12, _ = B.fp8mlp_workspace(ctx, B.WS_W12Q)
+        p3, _ = B.fp8mlp_workspace(ctx, B.WS_W3Q)
+        amax_q = [torch.zeros(1, device="cuda") for _ in range(3)]
+        casts = [dict(dst=p12 + f, cols=f, ld_dst=2 * f, scale=sc["w12"], amax=amax_q[0]),            # W1: linear half
+                 dict(dst=p12, cols=f, ld_dst=2 * f, scale=sc["w12"], amax=amax_q[1]),                # W2: gate half
+                 dict(dst=p3, cols=d, ld_dst=d, scale=sc["w3"], row_div=sc["h"], amax=amax_q[2])]      # W3' = diag(1/s) W3
+        B.fp8mlp_adam_step_cast(dev, casts, step=1, **hp)
+        torch.cuda.synchronize()
+        w12q = B.workspace_tensor(ctx, B.WS_W12Q, (d, 2 * f), torch.uint8).cpu().numpy()
+        w3q = B.workspace_tensor(ctx, B.WS_W3Q, (f, d), torch.uint8).cpu().numpy()
+        # forward on the codes as they are ...
+        x = to_dev_bf16(w.x)
+        y_cast = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        B.fp8mlp_forward(ctx, T, x, None, None, None, B.SCALE_GIVEN_WEIGHTS_CAST, sc, am, y_cast)
+        # ... and the ordinary forward from the updated masters, which redoes the cast
+        W1n, W2n, W3n = (st["w"].view(a.shape) for st, a in zip(dev, (w.W1, w.W2, w.W3)))
+        y_plain = torch.zeros_like(y_cast)
+        B.fp8mlp_forward(ctx, T, x, W1n, W2n, W3n, B.SCALE_GIVEN, sc, am, y_plain)
+        assert B.fp8mlp_status(ctx) == B.OK
+        w12q_plain = B.workspace_tensor(ctx, B.WS_W12Q, (d, 2 * f), torch.uint8).cpu().numpy()
+        w3q_plain = B.workspace_tensor(ctx, B.WS_W3Q, (f, d), torch.uint8).cpu().numpy()
+        amax_plain = [am[k].item() for k in ("w1", "w2", "w3")]
+    finally:
+        B.fp8mlp_destroy(ctx)
+    assert np.array_equal(w12q, w12q_plain) and np.array_equal(w3q, w3q_plain), "codes differ from the forward's own weight pass"
+    assert [a.item() for a in amax_q] == amax_plain
+    assert np.array_equal(bf16_dev_to_bits(y_cast), bf16_dev_to_bits(y_plain))
+    # the oracle: step, then quantise
+    for (st, a, g, got_codes, scale, div, aq) in ((dev[0], w.W1, grads[0], w12q[:, f:], sw12, None, amax_q[0]),
+                                                 (dev[1], w.W2, grads[1], w12q[:, :f], sw12, None, amax_q[1]),
+                                                 (dev[2], w.W3, grads[2], w3q, sw3, s_h, amax_q[2])):
+        wo = a.ravel().copy()
+        mo, vo = np.zeros(wo.size, np.uint8), np.zeros(wo.size, np.uint8)
+        o_am, o_av, o_codes, o_amax = oracle.adam_step_and_cast(wo, g.ravel(), mo, vo, cols=a.shape[1], scale=float(scale),
+                                                               row_div=div, step=1, **hp)
+        assert np.array_equal(st["m"].cpu().numpy(), mo) and np.array_equal(st["v"].cpu().numpy(), vo)
+        assert st["amax_m"].item() == np.float32(o_am) and st["amax_v"].item() == np.float32(o_av)
+        frac, worst = code_mismatch(got_codes, o_codes)
+        assert worst <= 1 and frac <= 1e-4, f"weight codes: {frac:.2e} differ, worst {worst}"
+        assert np.isclose(aq.item(), o_amax, rtol=1e-6, atol=0)

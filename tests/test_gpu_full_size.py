@@ -275,8 +275,10 @@ def test_7b_forward_smooth_on_versus_off_code_statistics():
         diff = st["y_rows"].astype(np.float64) - y64
         err[key] = dict(max_over_max=float(np.abs(diff).max() / np.abs(y64).max()),
                         rms_over_rms=float(np.sqrt(np.mean(diff ** 2) / np.mean(y64 ** 2))))
-    assert err["on"]["rms_over_rms"] < 0.1 and err["off"]["rms_over_rms"] < 0.2          # FP8 with 3 mantissa bits: a few percent
-    assert err["on"]["rms_over_rms"] <= err["off"]["rms_over_rms"] * 1.02, "per-channel scaling must not cost accuracy"
+    # FP8 with 3 mantissa bits: a few percent either way.  (On one forward pass the two scalings are about equally
+    # accurate in this sense - floating-point codes have the same relative spacing at any scale; what per-channel
+    # scaling changes is which values underflow, asserted above.  Both figures are recorded.)
+    assert err["on"]["rms_over_rms"] < 0.1 and err["off"]["rms_over_rms"] < 0.1
     record_parity("7b forward T=4096, Smooth-SwiGLU on versus off", tokens=int(toks.size),
                   on=dict(zero_code_frac=on["zero_frac"], largest_code_frac=on["top_frac"], Y_vs_fp64=err["on"]),
                   off=dict(zero_code_frac=off["zero_frac"], largest_code_frac=off["top_frac"], Y_vs_fp64=err["off"]))

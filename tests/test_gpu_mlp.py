@@ -9,7 +9,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import (bf16_dev_to_bits, bf16_bits_to_f32, bf16_ulp, check_amax_dz, check_dz_codes, code_mismatch, nmax_err,
+from helpers import (bf16_dev_to_bits, bf16_bits_to_f32, bf16_ulp, check_amax_dz, check_dz_codes, code_diff, code_mismatch, nmax_err,
                      nmax_err_bf16, record_parity, to_dev, to_dev_bf16)
 from paper_2409_12517_b200 import binding as B
 from paper_2409_12517_b200 import workloads as wl
@@ -82,7 +82,12 @@ def check_forward(r: Run, fw: dict, save=True):
         for name, got, ref in (("G", r.GU[:, :f], fw["G"]), ("U", r.GU[:, f:], fw["U"])):
             e = nmax_err_bf16(got, bf16_bits_to_f32(ref))
             assert e <= 1e-5, f"saved {name}: {e} beyond one bf16 spacing"
-    e = nmax_err(bf16_bits_to_f32(r.Y_bits), fw["Y"])
+    # Y is contracted from the Hq codes: the few allowed one-step differences (a step is 6-12 % of that element) are
+    # carried through the oracle's own W3' codes and set aside; zero when the codes agree, so no excuse for the GEMM
+    dh = code_diff(oracle.E4M3, r.Hq, fw["Hq"])
+    dq2 = (np.float32(1.0) / np.float32(fw["sw3"])) * (np.float32(1.0) if r.smooth else np.float32(1.0) / fw["s_h"][0])
+    y_ref = fw["Y"] + (dh @ oracle.decode(oracle.E4M3, fw["W3q"]).astype(np.float64)) * float(dq2) if np.any(dh) else fw["Y"]
+    e = nmax_err(bf16_bits_to_f32(r.Y_bits), y_ref)
     assert e <= OUT_TOL, f"Y: {e}"
 
 
@@ -103,11 +108,26 @@ def check_backward(r: Run, fw: dict, bw: dict, many_codes: bool = False):
     else:
         frac, worst = code_mismatch(r.dZq, bw["dZq"])
         assert worst <= 1 and frac <= CODE_FRAC, f"dZq codes: {frac:.2e} differ, worst {worst} steps"
+    # Outputs contracted from codes that may differ by a step on a few elements (dX, dW1, dW2 from dZq; dW3 from Hq):
+    # with few tokens one such step is visible in a weight-gradient column.  That part is computed from the code
+    # differences and the oracle's other operand and set aside (zero where the codes agree); the rest meets the bar.
+    inv = lambda v: np.float64(np.float32(1.0) / np.float32(v))
+    dz = code_diff(oracle.E5M2, r.dZq, bw["dZq"])
+    dh = code_diff(oracle.E4M3, r.Hq, fw["Hq"])
+    shift = dict(dX=0.0, dW1=0.0, dW2=0.0, dW3=0.0)
+    if np.any(dz):
+        xq = oracle.decode(oracle.E4M3, fw["Xq"]).astype(np.float64)
+        shift["dX"] = (dz @ oracle.decode(oracle.E4M3, fw["W12q"]).astype(np.float64).T) * inv(bw["sdz"]) * inv(fw["sw12"])
+        shift["dW2"] = (xq.T @ dz[:, :f]) * inv(fw["sx"]) * inv(bw["sdz"])
+        shift["dW1"] = (xq.T @ dz[:, f:]) * inv(fw["sx"]) * inv(bw["sdz"])
+    if np.any(dh):
+        dyq = oracle.decode(oracle.E5M2, bw["dYq"]).astype(np.float64)
+        shift["dW3"] = (dh.T @ dyq) * inv(bw["sdy"]) * (1.0 / fw["s_h"].astype(np.float64))[:, None]
     for name, got, ref in (("dX", bf16_bits_to_f32(r.dX_bits), bw["dX"]), ("dW1", r.dW1.cpu().numpy(), bw["dW1"]),
                            ("dW2", r.dW2.cpu().numpy(), bw["dW2"]), ("dW3", r.dW3.cpu().numpy(), bw["dW3"])):
         assert np.all(np.isfinite(got)), f"{name} has unwritten or non-finite entries"
-        e = nmax_err(got, ref)
-        assert e <= OUT_TOL, f"{name}: {e}"
+        e = nmax_err(got, ref + shift[name])
+        assert e <= OUT_TOL, f"{name}: {e} (literal {nmax_err(got, ref)})"
 
 
 def _oracle_flags(flags):
@@ -129,10 +149,15 @@ def test_tiny_config_current_amax(flags):
         r.close()
 
 
-@pytest.mark.parametrize("shape", [(200, 320, 272), (1, 16, 16), (130, 144, 528), (333, 512, 1040)])
+@pytest.mark.parametrize("shape", [(200, 320, 272), (1, 16, 16), (130, 144, 528), (333, 512, 1040), (300, 512, 2304),
+                                   (2048, 256, 272)])
 def test_ragged_shapes_given_scales(shape):
     """Several tiles with ragged tails in every dimension, delayed-scaling mode: scales come from an
-    oracle run on other data (a previous step), so values also saturate and underflow."""
+    oracle run on other data (a previous step), so values also saturate and underflow.  The last shapes have
+    few output tiles and long contractions, so their GEMMs split the contraction over several CTA pairs:
+    (333, 512, 1040) the input-gradient GEMM in two; (300, 512, 2304) the down projection in two and the
+    input-gradient GEMM in four; (2048, 256, 272) both weight-gradient GEMMs (fp32 outputs, one with a per-row
+    divisor, one with its columns split over two outputs at a column that is no multiple of 32)."""
     T, d, f = shape
     w = wl.make("r", 11, T, d, f, w_std=0.05, channel_outlier_frac=0.01, token_outlier_frac=0.02)
     prev = wl.make("p", 12, T, d, f, w_std=0.05)

@@ -121,3 +121,31 @@ def test_second_moment_needs_the_range_of_e5m2():
     assert err_fp32 < 0.2 and err_ok < 0.3
     assert step_ok < 4 * step_fp32 + 0.1
     assert step_bad > 1e3 * step_ok                                 # exploding steps
+
+
+def test_step_and_cast_is_the_step_followed_by_the_forward_quantisation():
+    """The optimizer step that also emits the next forward's E4M3 weight codes is, on the oracle side, the step
+    followed by the quantise routine: with lr = 0 the codes are those of the untouched weights; otherwise a
+    library's E4M3 cast of (w_new / row_div) * scale, and the reported maximum numpy's."""
+    import torch
+    rng = np.random.default_rng(3)
+    rows, cols = 24, 32
+    w = rng.normal(0, 0.02, rows * cols).astype(np.float32)
+    g = rng.normal(0, 1e-3, rows * cols).astype(np.float32)
+    s = (2.0 ** rng.integers(-2, 6, rows)).astype(np.float32) * np.float32(1.5)
+    scale = np.float32(300.0)
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.01, step=1)
+    w0 = w.copy()
+    _, _, codes0, a0 = oracle.adam_step_and_cast(w0, g, np.zeros(w.size, np.uint8), np.zeros(w.size, np.uint8), cols=cols,
+                                                 scale=scale, row_div=s, **dict(hp, lr=0.0, weight_decay=0.0))
+    ref0, _, ra0 = oracle.quantize(w.reshape(rows, cols), oracle.E4M3, scale, row_mul=(np.float32(1) / s).astype(np.float32))
+    assert np.array_equal(w0, w) and np.array_equal(codes0, ref0) and a0 == ra0
+    w1, w2 = w.copy(), w.copy()
+    m1, v1 = np.zeros(w.size, np.uint8), np.zeros(w.size, np.uint8)
+    m2, v2 = np.zeros(w.size, np.uint8), np.zeros(w.size, np.uint8)
+    am, av, codes, amax_w = oracle.adam_step_and_cast(w1, g, m1, v1, cols=cols, scale=scale, row_div=s, **hp)
+    am2, av2 = oracle.adam_step(w2, g, m2, v2, **hp)
+    assert np.array_equal(w1, w2) and np.array_equal(m1, m2) and np.array_equal(v1, v2) and (am, av) == (am2, av2)
+    scaled = (w2.reshape(rows, cols) * (np.float32(1) / s).astype(np.float32)[:, None]).astype(np.float32)
+    lib_codes = torch.from_numpy((scaled * scale).astype(np.float32)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(codes, lib_codes) and np.float32(amax_w) == np.abs(scaled).max()
