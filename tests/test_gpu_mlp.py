@@ -298,3 +298,33 @@ def test_empty_inputs_of_the_other_entry_points():
     finally:
         B.fp8mlp_destroy(ctx)
         B.fp8mlp_destroy(hb)
+
+
+def test_split_contraction_gives_the_same_bits_every_time():
+    """GEMMs with few tiles split their contraction over several CTA pairs and the share that finishes last
+    adds the partial sums - always in the order of the shares, so which one is last must not show in the result."""
+    T, d, f = 300, 512, 2304
+    w = wl.make("det", 23, T, d, f, w_std=0.05)
+    ctx = B.fp8mlp_create(T, d, f, B.SMOOTH | B.SAVE_FOR_BWD)
+    try:
+        sc, am = B.new_scales(f), B.new_amax(f)
+        x, dy = to_dev_bf16(w.x), to_dev_bf16(w.dY)
+        W1, W2, W3 = to_dev(w.W1), to_dev(w.W2), to_dev(w.W3)
+        y = torch.zeros((T, d), dtype=torch.bfloat16, device="cuda")
+        dx = torch.zeros_like(y)
+        dW1, dW2, dW3 = torch.zeros_like(W1), torch.zeros_like(W2), torch.zeros_like(W3)
+        B.fp8mlp_forward(ctx, T, x, W1, W2, W3, B.SCALE_FROM_CURRENT_AMAX, sc, am, y)
+        B.fp8mlp_backward(ctx, T, dy, B.SCALE_FROM_CURRENT_AMAX, sc, am, dx, dW1, dW2, dW3)
+        first = None
+        for _ in range(6):
+            B.fp8mlp_forward(ctx, T, x, W1, W2, W3, B.SCALE_GIVEN, sc, am, y)
+            B.fp8mlp_backward(ctx, T, dy, B.SCALE_GIVEN, sc, am, dx, dW1, dW2, dW3)
+            torch.cuda.synchronize()
+            got = [t.view(torch.int16).clone() for t in (y, dx)] + [t.view(torch.int32).clone() for t in (dW1, dW2, dW3)]
+            if first is None:
+                first = got
+            else:
+                assert all(torch.equal(a, b) for a, b in zip(got, first))
+        assert B.fp8mlp_status(ctx) == B.OK
+    finally:
+        B.fp8mlp_destroy(ctx)
