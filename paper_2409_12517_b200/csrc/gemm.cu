@@ -629,15 +629,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             bool ok = true;
             const CUtensorMap* tmB = (PAIR && rank != 0) ? &tmB1 : &tmB0;
             const uint64_t pol_a = l2_policy(p.hint_a), pol_b = l2_policy(p.hint_b);
-            for (int item = first_tile; ok && item < num_tiles; item += tile_step) {
+            int it = 0;
+            for (int item = first_tile; ok && item < num_tiles; item += tile_step, ++it) {
                 int m_tile, n_tile;
                 const int tile = item / p.split_k, split = item - tile * p.split_k;
                 tile_coords(p, tile, m_tile, n_tile);
                 const int m0 = m_tile * kTileM + static_cast<int>(rank) * kBlockM;
                 const int nb0 = n_tile * p.n_tile_cols + (PAIR ? static_cast<int>(rank) * p.b1_offset : 0);
                 const int nb1 = nb0 + p.b1_offset;
-                const int kb_end = min(p.num_k_blocks, (split + 1) * p.kb_per_split);
-                for (int kb = split * p.kb_per_split; kb < kb_end; ++kb) {
+                const int kb_begin = split * p.kb_per_split, kb_end = min(p.num_k_blocks, kb_begin + p.kb_per_split);
+                // Every other wave of tiles (a CTA's it-th tile belongs to the it-th wave) walks the contraction
+                // backwards: what L2 still holds when a wave ends is the end of the contraction, so the next wave meets
+                // the operand slice it shares with this one where it is still cached.  Only the order of the fp32 sum
+                // changes, and it is the same in every launch of the same problem.
+                const bool backwards = p.k_alternate && (it & 1);
+                for (int step = kb_begin; step < kb_end; ++step) {
+                    const int kb = backwards ? kb_begin + kb_end - 1 - step : step;
                     if (!mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     const uint32_t dst = tiles_addr + stage * kStageBytes;
                     const int k0 = kb * (kBlockK / ELEM);          // in elements
@@ -1057,6 +1064,7 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
     int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
     if (tiles == 0 || args.num_k_blocks == 0) return FP8MLP_OK;
     // A problem with fewer tiles than CTA pairs leaves SMs idle through a long contraction: split it.
+    args.k_alternate = 1;
     args.split_k = 1;
     args.kb_per_split = args.num_k_blocks;
     if (pair && !widen && (epi == EPI_F32 || epi == EPI_BF16) && args.partial != nullptr && args.tile_counters != nullptr) {

@@ -71,6 +71,7 @@ struct GemmArgs {
     float* out_f32_1;
     int n_split;
     int64_t ld_out;
+    int k_alternate;        // set by the launcher: every other wave of tiles walks the contraction backwards (L2 reuse)
     int tma_store;          // set by the launcher: the fp32 output leaves through shared memory and bulk tensor stores
     int stages;             // set by the launcher: operand stages in use (all of the kernel's, or two fewer when their
                             // shared memory stages the output)
