@@ -315,6 +315,24 @@ FP8MLP_API int fp8mlp_gemm_fp8(int64_t M, int64_t N, int64_t K,
                     const uint8_t* B, int b_kmajor, int b_fmt,
                     const float* scale_a, const float* scale_b, float* out, void* stream);
 
+/* How the library would run one of the block's GEMMs on a device with `sm_count` SMs: host arithmetic only, nothing
+ * is launched and no device is needed (for tests of the tiling rules and for tuning).  kind: 0 = fp32 output
+ * (weight gradients), 1 = bf16 output (down projection, input gradient), 2 = gate/up GEMM with the SwiGLU epilogue
+ * (N = d_ff), 3 = dgrad-2 with the SwiGLU-backward epilogue (N = d_ff).  with_workspace != 0: as inside a context
+ * (a split contraction is possible).  Returns FP8MLP_ERR_ARG for a bad kind or a null plan. */
+typedef struct {
+    int cta_pairs;          /* 1: 256-row tiles on CTA pairs (cta_group::2); 0: 128-row tiles on single CTAs      */
+    int tile_rows, tile_cols;
+    int m_tiles, n_tiles, k_stages;      /* k_stages: 128-byte steps of the contraction                            */
+    int split_k;            /* shares the contraction of a tile is cut into (1 = none)                             */
+    int stages_per_share;
+    int band_along_n, band_tiles;        /* rasterisation: bands of band_tiles tiles along m (0) or n (1)          */
+    int staged_stores;      /* fp32 output through shared memory and bulk tensor stores                            */
+    int64_t work_items;     /* tiles x split_k                                                                      */
+} fp8mlp_gemm_plan_t;
+FP8MLP_API int fp8mlp_gemm_plan(int kind, int64_t M, int64_t N, int64_t K, int sm_count, int with_workspace,
+                                fp8mlp_gemm_plan_t* plan);
+
 /* The same for bf16 operands (the unquantised last layer of FP8MLP_H_BF16 contexts): A, B bf16, no scales. */
 FP8MLP_API int fp8mlp_gemm_bf16(int64_t M, int64_t N, int64_t K, const void* A, int a_kmajor, const void* B,
                                 int b_kmajor, float* out, void* stream);

@@ -29,7 +29,7 @@ EXPORTS = [
     "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8", "fp8mlp_profile_enable", "fp8mlp_profile_read",
     "fp8mlp_forward_static", "fp8mlp_adam_step", "fp8mlp_scale_from_amax",
     "fp8mlp_merge_weights", "fp8mlp_forward_merged", "fp8mlp_gemm_bf16",
-    "fp8mlp_selftest_wait_timeout", "fp8mlp_adam_step_cast",
+    "fp8mlp_selftest_wait_timeout", "fp8mlp_adam_step_cast", "fp8mlp_gemm_plan",
 ]
 PHASES = ["quant_x", "quant_w12", "quant_w3", "gemm1_swiglu", "gemm2_down", "quant_dy", "dgrad2_swiglu_bwd",
           "wgrad3", "dgrad1", "wgrad12", "misc"]
@@ -55,6 +55,11 @@ class _AdamTensor(C.Structure):
     _fields_ = [("w", C.c_void_p), ("g", C.c_void_p), ("m", C.c_void_p), ("v", C.c_void_p), ("n", C.c_int64),
                 ("scale_m_in", C.c_void_p), ("scale_v_in", C.c_void_p), ("scale_m_out", C.c_void_p),
                 ("scale_v_out", C.c_void_p), ("amax_m", C.c_void_p), ("amax_v", C.c_void_p)]
+
+
+class _GemmPlan(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("cta_pairs", "tile_rows", "tile_cols", "m_tiles", "n_tiles", "k_stages", "split_k",
+                                       "stages_per_share", "band_along_n", "band_tiles", "staged_stores")] + [("work_items", C.c_int64)]
 
 
 class _AdamCast(C.Structure):
@@ -104,6 +109,7 @@ def lib():
                                        C.c_float, C.c_int64, C.c_void_p]
         L.fp8mlp_adam_step_cast.argtypes = [C.POINTER(_AdamTensor), C.POINTER(_AdamCast), C.c_int, C.c_float, C.c_float,
                                             C.c_float, C.c_float, C.c_float, C.c_int64, C.c_void_p]
+        L.fp8mlp_gemm_plan.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.POINTER(_GemmPlan)]
         L.fp8mlp_scale_from_amax.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         L.fp8mlp_profile_enable.argtypes = [C.c_void_p, C.c_int]
         L.fp8mlp_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -274,6 +280,16 @@ def fp8mlp_adam_step_cast(tensors: list, casts: list, lr: float, beta1: float, b
            "fp8mlp_adam_step_cast")
 
 
+GEMM_F32_OUT, GEMM_BF16_OUT, GEMM_SWIGLU_FWD, GEMM_SWIGLU_BWD = 0, 1, 2, 3
+
+
+def fp8mlp_gemm_plan(kind: int, M: int, N: int, K: int, sm_count: int = 148, with_workspace: bool = True) -> dict:
+    """How the library would tile and schedule one GEMM (host arithmetic only; works without a GPU)."""
+    p = _GemmPlan()
+    _check(lib().fp8mlp_gemm_plan(kind, M, N, K, sm_count, int(with_workspace), C.byref(p)), "fp8mlp_gemm_plan")
+    return {n: getattr(p, n) for n, _ in _GemmPlan._fields_}
+
+
 def fp8mlp_scale_from_amax(amax, fp8_fmt: int, scale) -> None:
     _check(lib().fp8mlp_scale_from_amax(_ptr(amax), fp8_fmt, _ptr(scale), _stream()), "fp8mlp_scale_from_amax")
 
@@ -317,3 +333,10 @@ def workspace_tensor(ctx: int, which: int, shape, dtype):
         return torch.empty(shape, dtype=dtype, device="cuda")
     raw = torch.as_tensor(_DeviceBytes(ptr, nbytes), device="cuda")
     return raw[:need].view(dtype).view(shape).clone()
+
+
+def workspace_fill(ctx: int, which: int, byte: int) -> None:
+    """Sets every byte of a workspace buffer (for tests: a poison pattern shows what a call failed to write)."""
+    ptr, nbytes = fp8mlp_workspace(ctx, which)
+    if nbytes:
+        torch.as_tensor(_DeviceBytes(ptr, nbytes), device="cuda").fill_(byte)

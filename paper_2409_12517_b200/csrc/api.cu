@@ -780,6 +780,26 @@ int fp8mlp_forward_static(int64_t T, int64_t d, int64_t f, uint32_t flags, const
     return fp8mlp_forward(&c, T, x, W1, W2, W3, mode, sc, am, y, stream);
 }
 
+int fp8mlp_gemm_plan(int kind, int64_t M, int64_t N, int64_t K, int sm_count, int with_workspace, fp8mlp_gemm_plan_t* out) {
+    if (out == nullptr || kind < EPI_F32 || kind > EPI_SWIGLU_BWD || sm_count < 1) return FP8MLP_ERR_ARG;
+    if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return FP8MLP_ERR_SHAPE;
+    GemmArgs a = base_args(nullptr, static_cast<int>(M), static_cast<int>(N), static_cast<int>(K));
+    if (kind == EPI_SWIGLU_FWD) { a.n_tile_cols = 128; a.b1_offset = 0; }
+    static float ws_stand_in;               // never dereferenced: planning only asks whether a workspace exists
+    static unsigned int cnt_stand_in;
+    if (with_workspace) { a.partial = &ws_stand_in; a.partial_floats = kSplitFloats; a.tile_counters = &cnt_stand_in; a.counter_words = kSplitWords; }
+    const GemmPlan p = plan_gemm(kind, a, sm_count);
+    out->cta_pairs = p.pair ? 1 : 0;
+    out->tile_rows = p.tile_m;
+    out->tile_cols = a.n_tile_cols;
+    out->m_tiles = a.num_m_tiles; out->n_tiles = a.num_n_tiles; out->k_stages = a.num_k_blocks;
+    out->split_k = a.split_k; out->stages_per_share = a.kb_per_split;
+    out->band_along_n = a.band_n; out->band_tiles = a.group;
+    out->staged_stores = a.tma_store;
+    out->work_items = p.items;
+    return FP8MLP_OK;
+}
+
 int fp8mlp_gemm_bf16(int64_t M, int64_t N, int64_t K, const void* A, int a_kmajor, const void* B, int b_kmajor,
                      float* out, void* stream) {
     if (A == nullptr || B == nullptr || out == nullptr) return FP8MLP_ERR_ARG;

@@ -254,7 +254,8 @@ __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk
 template <int PENDING>      // ... except for the PENDING most recent groups
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(PENDING) : "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// makes this thread's shared-memory writes visible to the bulk-copy engine
+// orders this thread's ordinary shared-memory accesses with what the bulk-copy engine does to the same memory
+// afterwards (its reads of what was written, its overwriting of what was read)
 __device__ __forceinline__ void fence_smem_to_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");

@@ -35,6 +35,11 @@ constexpr int kMaxStages = 6;
 // place of the last two operand stages, which a short contraction does not need (args.stages, args.tma_store).
 constexpr int kStoreBlockBytes = 32 * 128;
 constexpr int kStagesLentToStores = 2;
+// The 256 x 512-tile kernels with bf16 output (down projection, input gradient) do not overlap their epilogue with a
+// main loop, so what the epilogue costs is what its stores cost: they stage 32-row x 32-column bf16 blocks (2 KiB,
+// 64-byte swizzle), two per epilogue warp, in shared memory of their own (these kernels use four 48-KiB stages).
+constexpr int kStoreBlockBytesBf16 = 32 * 64;
+template <int EPI, bool WIDEN> struct OwnStoreBytes { static constexpr int value = (EPI == EPI_BF16 && WIDEN) ? (kEpiThreads / 32) * 2 * kStoreBlockBytesBf16 : 0; };
 
 template <bool FUSED>            // FUSED: the SwiGLU epilogues, which keep per-channel scales and maxima of the tile here
 struct __align__(8) SmemTailT {
@@ -54,9 +59,9 @@ template <int EPI> using TailOf = SmemTailT<EPI == EPI_SWIGLU_FWD || EPI == EPI_
 template <bool PAIR, int EPI, bool WIDEN>
 constexpr size_t smem_bytes() {
     return 1024 /*alignment slack*/ + size_t(Plan<PAIR, EPI, WIDEN>::kStages) * Plan<PAIR, EPI, WIDEN>::kStageBytes +
-           (EPI == EPI_SWIGLU_BWD ? size_t(kGuSlots) * kGuSlotBytes : 0) + sizeof(TailOf<EPI>);
+           (EPI == EPI_SWIGLU_BWD ? size_t(kGuSlots) * kGuSlotBytes : 0) + OwnStoreBytes<EPI, WIDEN>::value + sizeof(TailOf<EPI>);
 }
-static_assert(smem_bytes<true, EPI_F32, false>() <= 232448 && smem_bytes<false, EPI_F32, false>() <= 232448 &&
+static_assert(smem_bytes<true, EPI_BF16, true>() <= 232448 && smem_bytes<true, EPI_F32, false>() <= 232448 && smem_bytes<false, EPI_F32, false>() <= 232448 &&
               smem_bytes<true, EPI_SWIGLU_BWD, false>() <= 232448, "shared memory plan exceeds what a CTA can have");
 
 // ---------------------------------------------------------------- descriptors
@@ -331,6 +336,42 @@ __device__ __forceinline__ void epilogue_split(const GemmArgs& p, uint32_t taddr
     }
 }
 
+// bf16 output through shared memory (see kStoreBlockBytesBf16): the thread writes its row's 32 values as four 16-byte
+// pieces (piece j of row r at piece j ^ ((r >> 1) & 3): the 64-byte swizzle), one lane sends the block off as a bulk
+// tensor store; rows past M and columns past N are cut off by the tensor map.
+__device__ __forceinline__ void epilogue_bf16_staged(const GemmArgs& p, const CUtensorMap* out, uint32_t warp_stage_addr,
+                                                     uint32_t& blocks_sent, uint32_t taddr, int lane, int half, int row0, int n0,
+                                                     float dq) {
+#pragma unroll 1
+    for (int jj = 0; jj < 4; ++jj) {
+        const int j = 4 * half + jj;
+        const int c0 = n0 + 32 * j;
+        if (c0 >= p.N) break;
+        uint32_t r[32];
+        tmem_ld32(taddr + 32 * j, r);
+        tmem_ld_wait();
+        uint32_t w[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+            w[e] = cvt_bf16x2(__fmul_rn(__uint_as_float(r[2 * e]), dq), __fmul_rn(__uint_as_float(r[2 * e + 1]), dq));
+        const uint32_t block = warp_stage_addr + (blocks_sent & 1u) * kStoreBlockBytesBf16;
+        ++blocks_sent;
+        if (lane == 0) tma_store_wait_read<1>();           // the store that used this block last has read it
+        __syncwarp();
+        const uint32_t sw = static_cast<uint32_t>((lane >> 1) & 3);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            st_shared_v4(block + static_cast<uint32_t>(lane) * 64u + ((static_cast<uint32_t>(q) ^ sw) * 16u),
+                         w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+        fence_smem_to_async_proxy();
+        __syncwarp();
+        if (lane == 0) {
+            tma_store_2d(out, block, c0, row0);
+            tma_store_commit();
+        }
+    }
+}
+
 // 32 floats -> 32 FP8 codes (32 bytes) at dst; the second 16 only if `both`
 template <int FMT>
 __device__ __forceinline__ void store_fp8x32(uint8_t* dst, const float (&v)[32], bool both, bool wide) {
@@ -480,6 +521,19 @@ __device__ __forceinline__ bool epilogue_swiglu_bwd(const GemmArgs& p, SmemTail*
                     uq[i] = ld_shared_v4(rbase + kGuBoxBytes + off);
                 }
             }
+            // The slot goes back to the loader, whose refill writes it through the bulk-copy engine (the async proxy),
+            // while these reads are ordinary (generic-proxy) loads: the two are only ordered by a proxy fence.  Without
+            // it the refill now and then overwrote a 16-byte piece before a lane had read it - 8 wrong channels in one
+            // row, a few times per 10^9 pieces, found by repeating a step and comparing bits.  Consuming the loaded
+            // words first makes each lane hold its data before it fences.
+            if (gu8 || k == half) {
+                uint32_t seen = 0;
+#pragma unroll
+                for (int i = 0; i < (gu8 ? 2 : 4); ++i)
+                    seen ^= gq[i].x ^ gq[i].y ^ gq[i].z ^ gq[i].w ^ uq[i].x ^ uq[i].y ^ uq[i].z ^ uq[i].w;
+                asm volatile("" ::"r"(seen) : "memory");
+                fence_smem_to_async_proxy();
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tail->gu_empty[slot]));     // this warp is done with the slot
             ++gu_fill;
@@ -577,7 +631,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t gu_base = tiles_addr + kStages * kStageBytes;     // ring of saved G, U chunks (backward only)
     const uint32_t store_base = tiles_addr + static_cast<uint32_t>(p.stages) * kStageBytes;   // staging blocks of the fp32 output, if used
     using Tail = TailOf<EPI>;
-    Tail* tail = reinterpret_cast<Tail*>(tiles_ptr + size_t(kStages) * kStageBytes + kRingBytes);
+    const uint32_t own_store_base = gu_base + kRingBytes;            // staging blocks of the wide-tile bf16 output
+    Tail* tail = reinterpret_cast<Tail*>(tiles_ptr + size_t(kStages) * kStageBytes + kRingBytes + OwnStoreBytes<EPI, WIDEN>::value);
     const uint32_t n_stages = static_cast<uint32_t>(p.stages);
 
     const int warp = threadIdx.x >> 5;
@@ -789,8 +844,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             } else if constexpr (EPI == EPI_BF16) {
                 if (!WIDEN && p.split_k > 1)
                     epilogue_split<EPI_BF16>(p, taddr, lane, half, p.tile_counters + tile * 16 + rank * 8 + (warp - 2), split, m, n0, dq0);
-                else epilogue_bf16(p, taddr, half, m, n0, dq0);
-                if constexpr (WIDEN) epilogue_bf16(p, taddr + kBlockN, half, m, n0 + kBlockN, dq0);
+                else if (WIDEN && p.tma_store) {
+                    const uint32_t mine = own_store_base + static_cast<uint32_t>(warp - 2) * (2 * kStoreBlockBytesBf16);
+                    epilogue_bf16_staged(p, &tmG, mine, blocks_sent, taddr, lane, half, m - lane, n0, dq0);
+                    epilogue_bf16_staged(p, &tmG, mine, blocks_sent, taddr + kBlockN, lane, half, m - lane, n0 + kBlockN, dq0);
+                } else {
+                    epilogue_bf16(p, taddr, half, m, n0, dq0);
+                    if constexpr (WIDEN) epilogue_bf16(p, taddr + kBlockN, half, m, n0 + kBlockN, dq0);
+                }
             } else if constexpr (EPI == EPI_SWIGLU_FWD) {
                 epilogue_swiglu_fwd<GU8>(p, tail, taddr, lane, half, m, n0, dq0, sgu, gu_max);
             } else {
@@ -815,7 +876,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 // others touch them again only after the next tile's barrier: no second barrier needed
             }
         }
-        if constexpr (EPI == EPI_F32) {
+        if constexpr (EPI == EPI_F32 || EPI == EPI_BF16) {
             if (lane == 0) tma_store_wait_all();       // the staged output has reached global memory
         }
         if constexpr (EPI == EPI_SWIGLU_BWD) {
@@ -868,8 +929,8 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
                 int64_t tiles, int sm_count, cudaStream_t st) {
     constexpr size_t kSmem = smem_bytes<PAIR, EPI, WIDEN>();
     GemmArgs args = args_in;
-    if (EPI != EPI_F32 || WIDEN) args.tma_store = 0;
-    args.stages = Plan<PAIR, EPI, WIDEN>::kStages - (args.tma_store ? kStagesLentToStores : 0);
+    if (!((EPI == EPI_F32 && !WIDEN) || (EPI == EPI_BF16 && WIDEN))) args.tma_store = 0;
+    args.stages = Plan<PAIR, EPI, WIDEN>::kStages - ((args.tma_store && EPI == EPI_F32) ? kStagesLentToStores : 0);
     // the saved activations [M, 2f] bf16 as two matrices of f columns: G, and U starting f elements in
     CUtensorMap tmG = tmA, tmU = tmA;
     if constexpr (EPI == EPI_SWIGLU_BWD) {
@@ -883,6 +944,13 @@ int launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB0, const CUtensorM
             if (rc == FP8MLP_OK) rc = make_tmap_ring(&tmU, args.gu + f, 2, f, rows, 4 * f);
         }
         if (rc != FP8MLP_OK) return rc;
+    }
+    if constexpr (EPI == EPI_BF16 && WIDEN) {
+        if (args.tma_store) {
+            int rc = make_tmap_out_bf16(&tmG, args.out_bf16, static_cast<uint64_t>(args.N), static_cast<uint64_t>(args.M),
+                                        static_cast<uint64_t>(args.ld_out) * 2);
+            if (rc != FP8MLP_OK) return rc;
+        }
     }
     if constexpr (EPI == EPI_F32 && !WIDEN) {
         if (args.tma_store) {                // the two outputs of a (possibly split) fp32 result, boxes of 32 x 32
@@ -986,6 +1054,23 @@ int make_tmap_ring(CUtensorMap* map, const void* base, int elem_bytes, uint64_t 
     return FP8MLP_OK;
 }
 
+int make_tmap_out_bf16(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return FP8MLP_ERR_CUDA;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {row_stride_bytes};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t elem[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_cuda_error_str("cuTensorMapEncodeTiled", "driver rejected the output tensor map");
+        return FP8MLP_ERR_CUDA;
+    }
+    return FP8MLP_OK;
+}
+
 int make_tmap_out_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return FP8MLP_ERR_CUDA;
@@ -1007,8 +1092,8 @@ int make_tmap_u8(CUtensorMap* map, const void* base, uint64_t inner, uint64_t ou
     return make_tmap(map, base, 1, false, inner, outer, row_stride);
 }
 
-int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUtensorMap& tmA, const CUtensorMap& tmB0,
-                const CUtensorMap& tmB1, GemmArgs args, int sm_count, cudaStream_t st) {
+GemmPlan plan_gemm(int epi, GemmArgs& args, int sm_count) {
+    GemmPlan plan{};
     // a CTA pair works on 256 rows at a time; a problem of at most 128 rows runs on single CTAs
     const bool pair = args.pair_mode == 1 || (args.pair_mode == 0 && args.M > kBlockM);
     const int tile_m = pair ? 2 * kBlockM : kBlockM;
@@ -1043,6 +1128,42 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
             args.group = static_cast<int>((along + bands - 1) / bands);
         }
     }
+    // fp32 outputs leave as bulk tensor stores when every box is at least as wide as the output is (32 columns)
+    // (and when the contraction is so short that the kernel is bound by its output: at 16 stages' worth of work and
+    // beyond, direct stores hide behind the main loop and the staging only costs shared-memory bandwidth)
+    args.tma_store = (epi == EPI_F32 && !widen && args.num_k_blocks <= 8 && args.N >= 32 &&
+                      (args.n_split >= args.N || (args.n_split >= 32 && args.N - args.n_split >= 32))) ? 1 : 0;
+    // the bf16 output of the 256 x 512-tile kernels always does: their epilogue is not hidden behind a main loop
+    if (epi == EPI_BF16 && widen) args.tma_store = 1;
+    int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
+    // A problem with fewer tiles than CTA pairs leaves SMs idle through a long contraction: split it.
+    args.k_alternate = 1;
+    args.split_k = 1;
+    args.kb_per_split = args.num_k_blocks;
+    if (tiles > 0 && args.num_k_blocks > 0 && pair && !widen && (epi == EPI_F32 || epi == EPI_BF16) && args.partial != nullptr &&
+        args.tile_counters != nullptr) {
+        const int64_t pairs = sm_count / 2;
+        int64_t want = pairs / tiles;                                   // shares per tile that still fit one wave
+        if (want > 8) want = 8;
+        while (want > 1 && args.num_k_blocks / want < 8) --want;        // a share keeps at least 8 stages' worth of work
+        while (want > 1 && want * static_cast<int64_t>(args.M) * args.N > args.partial_floats) --want;
+        if (want > 1 && tiles * 16 <= args.counter_words) {
+            args.kb_per_split = static_cast<int>((args.num_k_blocks + want - 1) / want);
+            args.split_k = (args.num_k_blocks + args.kb_per_split - 1) / args.kb_per_split;   // every share non-empty
+            tiles *= args.split_k;
+        }
+    }
+    plan.pair = pair; plan.widen = widen; plan.tile_m = tile_m; plan.items = tiles;
+    return plan;
+}
+
+int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUtensorMap& tmA, const CUtensorMap& tmB0,
+                const CUtensorMap& tmB1, GemmArgs args, int sm_count, cudaStream_t st) {
+    const GemmPlan plan = plan_gemm(epi, args, sm_count);
+    const bool pair = plan.pair, widen = plan.widen;
+    const int tile_m = plan.tile_m;
+    const int elem = args.elem_bytes == 2 ? 2 : 1;
+    const int64_t tiles = plan.items;
     // instruction descriptor: [4,6) D = fp32; [7,10) A format; [10,13) B format (0 = E4M3, 1 = E5M2);
     // bit 15 / 16: A / B is MN-major; [17,23) N >> 3; [24,29) M >> 4 (M counts both CTAs of a pair)
     args.idesc = (1u << 4) | (static_cast<uint32_t>(a_fmt) << 7) | (static_cast<uint32_t>(b_fmt) << 10) |
@@ -1056,29 +1177,7 @@ int launch_gemm(int epi, bool a_mn, bool b_mn, int a_fmt, int b_fmt, const CUten
         case EPI_SWIGLU_FWD: args.wide = al32(args.hq) && al32(args.gu8) && args.N % 32 == 0; break;
         default: args.wide = al32(args.dzq) && args.N % 32 == 0; break;
     }
-    // fp32 outputs leave as bulk tensor stores when every box is at least as wide as the output is (32 columns)
-    // (and when the contraction is so short that the kernel is bound by its output: at 16 stages' worth of work and
-    // beyond, direct stores hide behind the main loop and the staging only costs shared-memory bandwidth)
-    args.tma_store = (epi == EPI_F32 && !widen && args.num_k_blocks <= 8 && args.N >= 32 &&
-                      (args.n_split >= args.N || (args.n_split >= 32 && args.N - args.n_split >= 32))) ? 1 : 0;
-    int64_t tiles = static_cast<int64_t>(args.num_m_tiles) * args.num_n_tiles;
     if (tiles == 0 || args.num_k_blocks == 0) return FP8MLP_OK;
-    // A problem with fewer tiles than CTA pairs leaves SMs idle through a long contraction: split it.
-    args.k_alternate = 1;
-    args.split_k = 1;
-    args.kb_per_split = args.num_k_blocks;
-    if (pair && !widen && (epi == EPI_F32 || epi == EPI_BF16) && args.partial != nullptr && args.tile_counters != nullptr) {
-        const int64_t pairs = sm_count / 2;
-        int64_t want = pairs / tiles;                                   // shares per tile that still fit one wave
-        if (want > 8) want = 8;
-        while (want > 1 && args.num_k_blocks / want < 8) --want;        // a share keeps at least 8 stages' worth of work
-        while (want > 1 && want * static_cast<int64_t>(args.M) * args.N > args.partial_floats) --want;
-        if (want > 1 && tiles * 16 <= args.counter_words) {
-            args.kb_per_split = static_cast<int>((args.num_k_blocks + want - 1) / want);
-            args.split_k = (args.num_k_blocks + args.kb_per_split - 1) / args.kb_per_split;   // every share non-empty
-            tiles *= args.split_k;
-        }
-    }
 
 #define FP8MLP_DISPATCH_WIDE(E, AM, BM)                                                                     \
     if (widen && epi == E && a_mn == AM && b_mn == BM)                                                      \

@@ -108,6 +108,13 @@ int make_tmap(CUtensorMap* map, const void* base, int elem_bytes, bool mn_major,
 int make_tmap_ring(CUtensorMap* map, const void* base, int elem_bytes, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes);
 // Tensor map of an fp32 output matrix for bulk stores: boxes of 32 columns x 32 rows, 128-byte swizzle.
 int make_tmap_out_f32(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes);
+// The same for a bf16 output matrix: boxes of 32 columns x 32 rows, 64-byte swizzle.
+int make_tmap_out_bf16(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t row_stride_bytes);
+
+// How a GEMM will be run: fills in the tiling, rasterisation, split and output-path fields of `args` (all host
+// arithmetic, nothing is launched) and returns the rest.  launch_gemm starts with this.
+struct GemmPlan { bool pair, widen; int tile_m; int64_t items; };
+GemmPlan plan_gemm(int epi, GemmArgs& args, int sm_count);
 
 // Launches one GEMM.  a_mn / b_mn: the operand is MN-major.  The tensor maps describe A, and the
 // two 128-wide halves of the B tile (the same map twice unless they come from different matrices).

@@ -76,7 +76,10 @@ def check_dz_codes(name, got, ref, code_frac=1e-3, out_tol=2e-3):
         many = float(np.mean(np.abs(code_rank(got) - code_rank(ref)) > 1))
         assert many <= 2e-5, f"{name}: {many:.2e} of the codes differ by more than one step"
         dv, rv = oracle.decode(oracle.E5M2, got), oracle.decode(oracle.E5M2, ref)
-        assert nmax_err(dv, rv) <= out_tol, f"{name}: decoded difference {nmax_err(dv, rv)}"
+        far = np.argwhere(np.abs(code_rank(got) - code_rank(ref)) > 1)
+        worst_at = np.unravel_index(np.argmax(np.abs(dv.astype(np.float64) - rv)), dv.shape)
+        assert nmax_err(dv, rv) <= out_tol, (f"{name}: decoded difference {nmax_err(dv, rv)} at {worst_at}: got {dv[worst_at]} "
+                                             f"ref {rv[worst_at]}, max |ref| {np.abs(rv).max()}; {len(far)} codes beyond one step, first at {far[:8].tolist()}")
 
 
 def amax_dz_bounds(g, u, dh, g_step, u_step):

@@ -91,3 +91,42 @@ def test_binding_constants_match_the_header():
     assert [n for n, _ in B._Scales._fields_] == members("fp8mlp_scales")
     assert [n for n, _ in B._Amax._fields_] == members("fp8mlp_amax")
     assert C.sizeof(B._Scales) == 8 * len(B._Scales._fields_)
+
+
+def test_gemm_plans_at_the_benchmark_shapes():
+    """Host logic of the GEMM launcher (tiling, rasterisation, split contraction, staged stores), asked through the
+    C ABI without a device, at the 7B shape for the token counts of the benchmark's sweep."""
+    from paper_2409_12517_b200 import binding as B
+    d, f, sms = 4096, 11008, 148
+    plan = lambda kind, M, N, K, **kw: B.fp8mlp_gemm_plan(kind, M, N, K, sms, **kw)
+    # T = 16384: CTA pairs everywhere; the bf16-output GEMMs on 256 x 512 tiles; nothing split, nothing staged
+    T = 16384
+    g1, g2 = plan(B.GEMM_SWIGLU_FWD, T, f, d), plan(B.GEMM_BF16_OUT, T, d, f)
+    assert (g1["cta_pairs"], g1["tile_rows"], g1["tile_cols"], g1["m_tiles"], g1["n_tiles"], g1["k_stages"]) == (1, 256, 128, 64, 86, 32)
+    assert (g2["tile_cols"], g2["n_tiles"], g2["k_stages"], g2["split_k"], g2["staged_stores"]) == (512, 8, 86, 1, 0)
+    # rasterisation: bands along the smaller operand, cut so that a band's slice stays under 46 MB
+    assert (g2["band_along_n"], g2["band_tiles"]) == (1, 8)                                     # all of W3' (45 MB)
+    w3, d1, w12 = plan(B.GEMM_F32_OUT, f, d, T), plan(B.GEMM_BF16_OUT, T, d, 2 * f), plan(B.GEMM_F32_OUT, d, 2 * f, T)
+    assert (w3["band_along_n"], w3["band_tiles"]) == (1, 8) and (d1["band_along_n"], d1["band_tiles"]) == (1, 4)
+    assert (w12["band_along_n"], w12["band_tiles"]) == (0, 8) and w12["work_items"] == 16 * 86
+    assert (g1["band_along_n"], g1["band_tiles"]) == (0, 16)                                     # fused epilogues: 16 row tiles
+    # T = 512: 32 tiles for 74 CTA pairs -> the long contractions are split in two; the weight gradients (4 stages of
+    # work per tile) stage their output; without a context's workspace nothing is split
+    T = 512
+    g2, d1 = plan(B.GEMM_BF16_OUT, T, d, f), plan(B.GEMM_BF16_OUT, T, d, 2 * f)
+    assert (g2["tile_cols"], g2["m_tiles"] * g2["n_tiles"], g2["split_k"], g2["stages_per_share"], g2["work_items"]) == (256, 32, 2, 43, 64)
+    assert (d1["split_k"], d1["stages_per_share"]) == (2, 86)
+    assert plan(B.GEMM_BF16_OUT, T, d, f, with_workspace=False)["split_k"] == 1
+    w3, w12 = plan(B.GEMM_F32_OUT, f, d, T), plan(B.GEMM_F32_OUT, d, 2 * f, T)
+    assert w3["k_stages"] == 4 and w3["staged_stores"] == 1 and w12["staged_stores"] == 1 and w3["split_k"] == 1
+    assert plan(B.GEMM_F32_OUT, f, d, 2048)["staged_stores"] == 0                                # 16 stages: direct stores
+    assert plan(B.GEMM_SWIGLU_BWD, T, f, d)["split_k"] == 1                                       # fused epilogues never split
+    # every share of a split contraction is non-empty and the shares cover it
+    for K in (1024, 1152, 2304, 4608, 11008, 22016, 100000):
+        p = plan(B.GEMM_BF16_OUT, 256, 256, K)
+        assert (p["split_k"] - 1) * p["stages_per_share"] < p["k_stages"] <= p["split_k"] * p["stages_per_share"]
+        assert p["split_k"] == 1 or p["stages_per_share"] >= 8
+    # at most 128 rows: single CTAs with 128-row tiles
+    s = plan(B.GEMM_BF16_OUT, 128, 4096, 4096)
+    assert (s["cta_pairs"], s["tile_rows"]) == (0, 128)
+    assert B.lib().fp8mlp_gemm_plan(7, 16, 16, 16, 148, 0, None) == B.ERR_ARG
