@@ -327,7 +327,8 @@ typedef struct {
     int split_k;            /* shares the contraction of a tile is cut into (1 = none)                             */
     int stages_per_share;
     int band_along_n, band_tiles;        /* rasterisation: bands of band_tiles tiles along m (0) or n (1)          */
-    int staged_stores;      /* fp32 output through shared memory and bulk tensor stores                            */
+    int staged_stores;      /* output through shared memory and bulk tensor stores (fp32: short contractions;      */
+                            /* bf16: 256 x 512 tiles)                                                              */
     int64_t work_items;     /* tiles x split_k                                                                      */
 } fp8mlp_gemm_plan_t;
 FP8MLP_API int fp8mlp_gemm_plan(int kind, int64_t M, int64_t N, int64_t K, int sm_count, int with_workspace,
