@@ -19,6 +19,7 @@ pytestmark = pytest.mark.gpu
     (16384, 4096, 11008, B.SMOOTH | B.SAVE_FOR_BWD | B.GU_FP8, 30),      # saved activations as E4M3 codes
     (512, 4096, 11008, B.SMOOTH | B.SAVE_FOR_BWD, 100),                  # split contractions, staged stores
     (2520, 4048, 1040, B.SAVE_FOR_BWD, 60),                              # ragged tiles, Smooth-SwiGLU off
+    (4096, 4096, 11008, B.SAVE_FOR_BWD | B.H_BF16, 30),                  # the last layer in bf16 (16-bit operand path)
 ])
 def test_step_is_bitwise_repeatable(T, d, f, flags, reps):
     gen = torch.Generator(device="cuda").manual_seed(T + f)
@@ -36,14 +37,15 @@ def test_step_is_bitwise_repeatable(T, d, f, flags, reps):
 
         def snapshot():
             ws = lambda which, shape, dt=torch.uint8: B.workspace_tensor(ctx, which, shape, dt)
-            return dict(Hq=ws(B.WS_HQ, (T, f)), GU=ws(B.WS_GU, (T, 2 * f), gu_dtype), dZq=ws(B.WS_DZQ, (T, 2 * f)),
+            h = ws(B.WS_HB, (T, f), torch.int16) if flags & B.H_BF16 else ws(B.WS_HQ, (T, f))
+            return dict(H=h, GU=ws(B.WS_GU, (T, 2 * f), gu_dtype), dZq=ws(B.WS_DZQ, (T, 2 * f)),
                         Y=y.view(torch.int16).clone(), dX=dx.view(torch.int16).clone(), dW1=dW1.view(torch.int32).clone(),
                         dW2=dW2.view(torch.int32).clone(), dW3=dW3.view(torch.int32).clone(),
                         maxima=torch.cat([v.view(-1) for v in am.values()]).view(torch.int32).clone())
 
         first = None
         for rep in range(reps):
-            for which in (B.WS_HQ, B.WS_GU, B.WS_DZQ):                    # nothing survives from the previous repetition
+            for which in (B.WS_HB if flags & B.H_BF16 else B.WS_HQ, B.WS_GU, B.WS_DZQ):   # nothing survives from the previous repetition
                 B.workspace_fill(ctx, which, 0x7F)
             B.fp8mlp_forward(ctx, T, x, W1, W2, W3, B.SCALE_GIVEN, sc, am, y)
             B.fp8mlp_backward(ctx, T, dy, B.SCALE_GIVEN, sc, am, dx, dW1, dW2, dW3)
