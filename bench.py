@@ -37,7 +37,7 @@ FP8_OVER_BF16 = 2.0          # nominal dense tensor-core ratio (4.5 vs 2.25 PFLO
 NOMINAL_FP8_TFLOPS = 4500.0
 # DRAM bytes per launch of the dominant kernel (gate/up GEMM + SwiGLU epilogue) measured by ncu
 # (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None until captured.
-NCU_TRAFFIC_BYTES = {"7b": 451_462_000 + 865_298_688}     # profiles/gemm_kernels_7b.txt, GEMM-1 launch (read + write)
+NCU_TRAFFIC_BYTES = {"7b": 537_238_000 + 868_014_336}     # profiles/gemm_kernels_7b.txt, GEMM-1 launch (read + write)
 
 
 def flops_step(T, d, f):
@@ -171,6 +171,10 @@ class ClockSampler:
         if self.how is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source (NVML binding and nvidia-smi both unavailable)"]}
         timed, whole = self.window(t0, t1), self.window(t_warm, t1)
+        if timed["samples"] == 0 and self.rows:          # a timed region shorter than the polling period: the sample nearest to it
+            t, mhz, watts, reasons = min(self.rows, key=lambda r: min(abs(r[0] - t0), abs(r[0] - t1)))
+            timed = {"samples": 1, "sm_mhz": mhz, "sm_mhz_min": mhz, "sm_mhz_max": mhz, "power_w_max": watts,
+                     "reasons": sorted(reasons), "sw_power_cap_samples": int("sw_power_cap" in reasons), "nearest_sample_s": round(min(abs(t - t0), abs(t - t1)), 4)}
         return {"sm_mhz": timed.get("sm_mhz"), "sm_max_mhz": self.max_mhz, "reasons": timed.get("reasons", []),
                 "samples": timed["samples"], "power_w_max": timed.get("power_w_max"), "timed_region": timed,
                 "warmup_and_timed": whole, "source": self.how}
@@ -344,11 +348,15 @@ def run_forward_only(args, rank: int, local_rank: int):
         jit_mean, jit_med = timed(B.SCALE_FROM_CURRENT_AMAX, min(args.steps, 50))
         fwd(B.SCALE_FROM_CURRENT_AMAX)
         assert B.fp8mlp_status(ctx) == B.OK
-        mag = B.workspace_tensor(ctx, B.WS_HQ, (T, f), torch.uint8) & 0x7F
+        hq = B.workspace_tensor(ctx, B.WS_HQ, (T, f), torch.uint8)
+        counts = torch.zeros(2, dtype=torch.int64, device="cuda")
+        B.fp8mlp_code_stats(hq, B.E4M3, counts)
+        n_zero, n_top = (int(v) for v in counts.tolist())
+        mag = hq & 0x7F
         rows["smooth_on" if smooth else "smooth_off"] = {
             "ms": round(mean_ms, 4), "ms_median": round(med_ms, 4), "tflops": round(flops / (mean_ms * 1e-3) / 1e12, 1),
             "just_in_time_ms": round(jit_mean, 4), "just_in_time_tflops_useful": round(flops / (jit_mean * 1e-3) / 1e12, 1),
-            "zero_code_frac": float((mag == 0).float().mean()), "largest_code_frac": float((mag == 0x7E).float().mean()),
+            "zero_code_frac": n_zero / (T * f), "largest_code_frac": n_top / (T * f),
             "channels_whose_top_code_is_in_the_top_binade": int((mag.max(dim=0).values >= 0x76).sum()),
             "gpu_launches": launches}
         B.fp8mlp_destroy(ctx)

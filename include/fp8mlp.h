@@ -315,6 +315,15 @@ FP8MLP_API int fp8mlp_gemm_fp8(int64_t M, int64_t N, int64_t K,
                     const uint8_t* B, int b_kmajor, int b_fmt,
                     const float* scale_a, const float* scale_b, float* out, void* stream);
 
+/* How a tensor of FP8 codes used its format's range (Section 4.3 motivates Smooth-SwiGLU with exactly this view of the
+ * SwiGLU output: ordinary channels lost to underflow next to outlier channels at the top of the range):
+ *   *zero_count = codes that are +0 or -0;  *top_count = codes at the largest finite magnitude (448 / 57344), which is
+ *   where the saturating cast puts every value beyond it.
+ * codes: device, [rows, cols] with row stride ld (cols, ld multiples of 16; 16-byte aligned), e.g. a context's
+ * FP8MLP_WS_HQ buffer; the two counters are 8-byte aligned device words, overwritten.  One pass, 1 byte read per code. */
+FP8MLP_API int fp8mlp_code_stats(const uint8_t* codes, int64_t rows, int64_t cols, int64_t ld, int fp8_fmt,
+                                 uint64_t* zero_count, uint64_t* top_count, void* stream);
+
 /* How the library would run one of the block's GEMMs on a device with `sm_count` SMs: host arithmetic only, nothing
  * is launched and no device is needed (for tests of the tiling rules and for tuning).  kind: 0 = fp32 output
  * (weight gradients), 1 = bf16 output (down projection, input gradient), 2 = gate/up GEMM with the SwiGLU epilogue

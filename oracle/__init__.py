@@ -145,6 +145,15 @@ def quantize(src, fmt: int, scale: float, row_mul=None, flags: int = 0):
     return codes, deq, float(a.value)
 
 
+def code_stats(fmt: int, codes) -> tuple:
+    """(number of zero codes, number of codes at the largest finite magnitude) of a 2-D uint8 array of FP8 codes."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    rows, cols = codes.shape
+    z, t = C.c_int64(0), C.c_int64(0)
+    lib().orc_code_stats(C.c_int(fmt), _p(codes), C.c_int64(rows), C.c_int64(cols), C.c_int64(cols), C.byref(z), C.byref(t))
+    return int(z.value), int(t.value)
+
+
 def gemm(A, B) -> np.ndarray:
     """C = A @ B in fp32 with sequential accumulation over the contraction index.
 

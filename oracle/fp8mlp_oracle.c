@@ -225,6 +225,22 @@ void orc_quantize(const float* src, int64_t rows, int64_t cols, const float* row
     if (amax_out) *amax_out = a;
 }
 
+/* How the range of a format was used by a tensor of codes (Section 4.3 looks at exactly this for the SwiGLU
+ * output: values lost to underflow next to values at the top of the range): the number of codes that are
+ * zero (+0 or -0) and the number at the largest finite magnitude (where the saturating cast puts everything
+ * beyond it).  codes is [rows, cols] with row stride ld. */
+void orc_code_stats(int fmt, const uint8_t* codes, int64_t rows, int64_t cols, int64_t ld, int64_t* zero, int64_t* top) {
+    const uint8_t top_code = fmt == ORC_E4M3 ? 0x7E : 0x7B;
+    int64_t z = 0, t = 0;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < cols; ++c) {
+            const uint8_t mag = codes[r * ld + c] & 0x7F;
+            if (mag == 0) ++z;
+            if (mag == top_code) ++t;
+        }
+    *zero = z; *top = t;
+}
+
 float orc_amax_rows(const float* src, int64_t rows, int64_t cols, const float* row_mul) {
     float a = 0.0f;
     for (int64_t r = 0; r < rows; ++r)

@@ -29,7 +29,7 @@ EXPORTS = [
     "fp8mlp_forward", "fp8mlp_backward", "fp8mlp_gemm_fp8", "fp8mlp_profile_enable", "fp8mlp_profile_read",
     "fp8mlp_forward_static", "fp8mlp_adam_step", "fp8mlp_scale_from_amax",
     "fp8mlp_merge_weights", "fp8mlp_forward_merged", "fp8mlp_gemm_bf16",
-    "fp8mlp_selftest_wait_timeout", "fp8mlp_adam_step_cast", "fp8mlp_gemm_plan",
+    "fp8mlp_selftest_wait_timeout", "fp8mlp_adam_step_cast", "fp8mlp_gemm_plan", "fp8mlp_code_stats",
 ]
 PHASES = ["quant_x", "quant_w12", "quant_w3", "gemm1_swiglu", "gemm2_down", "quant_dy", "dgrad2_swiglu_bwd",
           "wgrad3", "dgrad1", "wgrad12", "misc"]
@@ -109,6 +109,7 @@ def lib():
                                        C.c_float, C.c_int64, C.c_void_p]
         L.fp8mlp_adam_step_cast.argtypes = [C.POINTER(_AdamTensor), C.POINTER(_AdamCast), C.c_int, C.c_float, C.c_float,
                                             C.c_float, C.c_float, C.c_float, C.c_int64, C.c_void_p]
+        L.fp8mlp_code_stats.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         L.fp8mlp_gemm_plan.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.POINTER(_GemmPlan)]
         L.fp8mlp_scale_from_amax.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         L.fp8mlp_profile_enable.argtypes = [C.c_void_p, C.c_int]
@@ -278,6 +279,14 @@ def fp8mlp_adam_step_cast(tensors: list, casts: list, lr: float, beta1: float, b
         c.amax = d["amax"].data_ptr() if d.get("amax") is not None else None
     _check(lib().fp8mlp_adam_step_cast(arr, carr, len(tensors), lr, beta1, beta2, eps, weight_decay, step, _stream()),
            "fp8mlp_adam_step_cast")
+
+
+def fp8mlp_code_stats(codes, fp8_fmt: int, counts, ld: int | None = None) -> None:
+    """codes: 2-D uint8 CUDA tensor (row stride ld, default cols); counts: int64 CUDA tensor of 2 elements, receives
+    (zero codes, codes at the largest finite magnitude)."""
+    rows, cols = codes.shape
+    _check(lib().fp8mlp_code_stats(_ptr(codes), rows, cols, cols if ld is None else ld, fp8_fmt, C.c_void_p(counts.data_ptr()),
+                                   C.c_void_p(counts.data_ptr() + 8), _stream()), "fp8mlp_code_stats")
 
 
 GEMM_F32_OUT, GEMM_BF16_OUT, GEMM_SWIGLU_FWD, GEMM_SWIGLU_BWD = 0, 1, 2, 3

@@ -403,6 +403,19 @@ int fp8mlp_quantize(const void* src, int src_dtype, int64_t rows, int64_t cols, 
                              amax, sms, st);
 }
 
+int fp8mlp_code_stats(const uint8_t* codes, int64_t rows, int64_t cols, int64_t ld, int fp8_fmt, uint64_t* zero_count,
+                      uint64_t* top_count, void* stream) {
+    if (codes == nullptr || zero_count == nullptr || top_count == nullptr) return FP8MLP_ERR_ARG;
+    if (fp8_fmt != FP8MLP_E4M3 && fp8_fmt != FP8MLP_E5M2) return FP8MLP_ERR_ARG;
+    if (rows < 0 || cols < 0 || cols % 16 != 0 || ld < cols || ld % 16 != 0) return FP8MLP_ERR_SHAPE;
+    if (!aligned16(codes) || (reinterpret_cast<uintptr_t>(zero_count) & 7u) || (reinterpret_cast<uintptr_t>(top_count) & 7u)) return FP8MLP_ERR_ALIGN;
+    int dev = 0, sms = 0;
+    FP8MLP_CUDA_CHECK(cudaGetDevice(&dev));
+    FP8MLP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    return run_code_stats(codes, rows, cols, ld, fp8_fmt, reinterpret_cast<unsigned long long*>(zero_count),
+                          reinterpret_cast<unsigned long long*>(top_count), sms, static_cast<cudaStream_t>(stream));
+}
+
 int fp8mlp_scale_from_amax(const float* amax, int fp8_fmt, float* scale, void* stream) {
     if (amax == nullptr || scale == nullptr) return FP8MLP_ERR_ARG;
     if (fp8_fmt != FP8MLP_E4M3 && fp8_fmt != FP8MLP_E5M2) return FP8MLP_ERR_ARG;

@@ -231,6 +231,38 @@ __global__ void __launch_bounds__(kThreads) cast_bf16_kernel(const float* __rest
     if (amax_out != nullptr) block_atomic_max(local_max, amax_out);
 }
 
+// Zero codes and codes at the largest finite magnitude of an FP8 tensor [rows, cols] (row stride ld, both multiples
+// of 16): a unit is 16 codes; counts go to two 64-bit device counters.
+__global__ void __launch_bounds__(kThreads) code_stats_kernel(const uint8_t* __restrict__ codes, int64_t n_units, int units_per_row,
+                                                              int64_t ld, uint32_t top_code, unsigned long long* zero,
+                                                              unsigned long long* top) {
+    grid_dependency_wait();
+    grid_launch_dependents();
+    unsigned int z = 0, t = 0;
+    for (int64_t u = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; u < n_units;
+         u += static_cast<int64_t>(gridDim.x) * kThreads) {
+        const int64_t r = u / units_per_row, c = u - r * units_per_row;
+        const uint4 v = ld_global_nc_v4(codes + r * ld + c * 16);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t mag = w[i] & 0x7F7F7F7Fu;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const uint32_t m = (mag >> (8 * b)) & 0xFFu;
+                z += m == 0u;
+                t += m == top_code;
+            }
+        }
+    }
+    z = __reduce_add_sync(0xffffffffu, z);
+    t = __reduce_add_sync(0xffffffffu, t);
+    if ((threadIdx.x & 31) == 0) {
+        if (z) atomicAdd(zero, static_cast<unsigned long long>(z));
+        if (t) atomicAdd(top, static_cast<unsigned long long>(t));
+    }
+}
+
 template <typename SRC, int FMT>
 int launch_pass(bool cast, bool amax, const QuantLaunch& q, int grid, cudaStream_t st) {
     cudaError_t e;
@@ -317,6 +349,20 @@ int run_cast_bf16(const float* src, uint16_t* dst, int64_t n, float* amax_out, i
     int64_t blocks = (units + kThreads - 1) / kThreads;
     if (blocks > int64_t(sm_count) * 8) blocks = int64_t(sm_count) * 8;
     FP8MLP_CUDA_CHECK(launch_chained(cast_bf16_kernel, static_cast<int>(blocks), kThreads, 0, st, src, dst, units, amax_out));
+    FP8MLP_LAUNCH_CHECK();
+    return FP8MLP_OK;
+}
+
+int run_code_stats(const uint8_t* codes, int64_t rows, int64_t cols, int64_t ld, int fmt, unsigned long long* zero,
+                   unsigned long long* top, int sm_count, cudaStream_t st) {
+    FP8MLP_CUDA_CHECK(cudaMemsetAsync(zero, 0, sizeof(unsigned long long), st));
+    FP8MLP_CUDA_CHECK(cudaMemsetAsync(top, 0, sizeof(unsigned long long), st));
+    const int64_t units = rows * (cols / 16);
+    if (units == 0) return FP8MLP_OK;
+    int64_t blocks = (units + kThreads - 1) / kThreads;
+    if (blocks > int64_t(sm_count) * 8) blocks = int64_t(sm_count) * 8;
+    FP8MLP_CUDA_CHECK(launch_chained(code_stats_kernel, static_cast<int>(blocks), kThreads, 0, st, codes, units,
+                                     static_cast<int>(cols / 16), ld, fmt == FP8MLP_E4M3 ? 0x7Eu : 0x7Bu, zero, top));
     FP8MLP_LAUNCH_CHECK();
     return FP8MLP_OK;
 }

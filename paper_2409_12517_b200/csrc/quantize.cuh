@@ -37,6 +37,8 @@ int run_quantize_pass(bool cast, bool amax, const void* src, int src_dtype, int6
                       int sm_count, cudaStream_t st);
 
 // dst[i] = bf16(src[i]) (n % 8 == 0), *amax_out raised to max |src| (nullable; zeroed by the caller)
+int run_code_stats(const uint8_t* codes, int64_t rows, int64_t cols, int64_t ld, int fmt, unsigned long long* zero,
+                   unsigned long long* top, int sm_count, cudaStream_t st);
 int run_cast_bf16(const float* src, uint16_t* dst, int64_t n, float* amax_out, int sm_count, cudaStream_t st);
 
 // *scale = fmt_max / max(*amax_a, *amax_b)  (amax_b nullable), 1 for a zero / non-finite amax

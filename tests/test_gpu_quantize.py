@@ -128,3 +128,23 @@ def test_update_scales_matches_oracle(smooth):
         assert np.array_equal(got, ref)
     finally:
         B.fp8mlp_destroy(ctx)
+
+
+@pytest.mark.parametrize("fmt", [B.E4M3, B.E5M2])
+@pytest.mark.parametrize("shape,ld", [((1, 16), 16), ((333, 1040), 1040), ((700, 272), 544), ((4096, 11008), 11008)])
+def test_code_stats_match_the_oracle(fmt, shape, ld):
+    """fp8mlp_code_stats (zero codes, codes at the largest finite magnitude) against the oracle's counts, exactly; rows
+    may be strided (a column block of a wider buffer)."""
+    rng = np.random.default_rng(shape[0] + fmt)
+    full = rng.integers(0, 256, (shape[0], ld), dtype=np.uint8)
+    full[rng.random(full.shape) < 0.05] = 0x80                           # plenty of -0
+    full[rng.random(full.shape) < 0.01] = 0x7E if fmt == B.E4M3 else 0xFB  # and of the largest magnitude
+    dev = torch.from_numpy(full).cuda()
+    counts = torch.full((2,), -1, dtype=torch.int64, device="cuda")
+    L = B.lib()
+    import ctypes as C
+    rc = L.fp8mlp_code_stats(C.c_void_p(dev.data_ptr()), shape[0], shape[1], ld, fmt, C.c_void_p(counts.data_ptr()),
+                             C.c_void_p(counts.data_ptr() + 8), C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    assert rc == B.OK
+    torch.cuda.synchronize()
+    assert tuple(counts.tolist()) == oracle.code_stats(oracle.E4M3 if fmt == B.E4M3 else oracle.E5M2, full[:, :shape[1]])

@@ -530,3 +530,22 @@ def test_amax_dz_envelope_of_the_parity_tests():
     assert lo == hi and np.isclose(lo, bw["amax_dz"], rtol=1e-6)
     lo, hi = amax_dz_bounds(g, u, bw["dH"], bf16_ulp(g), bf16_ulp(u))
     assert lo <= bw["amax_dz"] <= hi and hi / lo < 1.0 + 8 * 2.0 ** -7
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E5M2])
+def test_code_stats_counts_zero_and_top_codes(fmt):
+    """Pins of the code statistics: among all 256 codes exactly two are zero (+0, -0) and two sit at the largest finite
+    magnitude; on random values the counts equal those a library cast's values give (value == 0, |value| == format
+    maximum); and a quantised tensor scaled to its own maximum has at least one top code and none beyond."""
+    allc = np.arange(256, dtype=np.uint8).reshape(16, 16)
+    assert oracle.code_stats(fmt, allc) == (2, 2)
+    rng = np.random.default_rng(11)
+    v = (rng.standard_normal((64, 48)) * rng.choice([1e-9, 1.0, 1e6], (64, 48))).astype(np.float32)
+    codes, deq, _ = oracle.quantize(v, fmt, 1.0)
+    tdt = torch.float8_e4m3fn if fmt == E4M3 else torch.float8_e5m2
+    lib_vals = torch.from_numpy(codes).view(tdt).float().numpy()
+    fmax = oracle.fmt_max(fmt)
+    assert oracle.code_stats(fmt, codes) == (int(np.sum(lib_vals == 0)), int(np.sum(np.abs(lib_vals) == fmax)))
+    assert oracle.code_stats(fmt, codes)[0] > 0 and oracle.code_stats(fmt, codes)[1] > 0      # the draw underflows and saturates
+    own = oracle.quantize(v, fmt, oracle.scale_from_amax(fmt, oracle.amax(v)))[0]
+    assert oracle.code_stats(fmt, own)[1] >= 1
