@@ -15,7 +15,11 @@
  *     16-byte aligned; the library never frees or reallocates them.  d and f must be
  *     multiples of 16 (FP8MLP_ERR_SHAPE otherwise); T is any value >= 0 and <= T_max.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
- *     enqueue work on it and return; nothing synchronises the device.
+ *     enqueue work on it and return; nothing synchronises the device.  The kernels are launched with
+ *     programmatic stream serialisation (each waits for its predecessor in the stream before it touches
+ *     global memory), which is invisible to the caller: the stream behaves as an in-order stream, and
+ *     work the caller enqueues before or after a call is ordered as usual.
+ *   - Results are deterministic: the same inputs, scales and shapes give the same bits in every call.
  *   - The return value is FP8MLP_OK (0) or a negative FP8MLP_ERR_* code.  Argument errors are
  *     detected before anything is launched.  Nothing throws or aborts across this boundary.
  *   - bf16 tensors are passed as void* (2 bytes per element); FP8 codes as uint8_t.
