@@ -62,3 +62,47 @@ def test_step_is_bitwise_repeatable(T, d, f, flags, reps):
         assert B.fp8mlp_status(ctx) == B.OK
     finally:
         B.fp8mlp_destroy(ctx)
+
+
+def test_just_in_time_step_and_merged_forward_are_bitwise_repeatable():
+    """The same for the step with every scale derived from the current data (calibration passes, scale kernels) and
+    for the inference form on merged weights."""
+    T, d, f = 4096, 4096, 11008
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    x = torch.randn(T, d, device="cuda", generator=gen).to(torch.bfloat16)
+    dy = (torch.randn(T, d, device="cuda", generator=gen) * 1e-3).to(torch.bfloat16)
+    W1, W2, W3 = (torch.randn(*s, device="cuda", generator=gen) * 0.02 for s in ((d, f), (d, f), (f, d)))
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    dW1, dW2, dW3 = torch.empty_like(W1), torch.empty_like(W2), torch.empty_like(W3)
+    ctx = B.fp8mlp_create(T, d, f, B.SMOOTH | B.SAVE_FOR_BWD)
+    try:
+        sc, am = B.new_scales(f), B.new_amax(f)
+        first = None
+        for rep in range(12):
+            for t in (y, dx, dW1, dW2, dW3):
+                t.fill_(float("nan"))
+            B.fp8mlp_forward(ctx, T, x, W1, W2, W3, B.SCALE_FROM_CURRENT_AMAX, sc, am, y)
+            B.fp8mlp_backward(ctx, T, dy, B.SCALE_FROM_CURRENT_AMAX, sc, am, dx, dW1, dW2, dW3)
+            torch.cuda.synchronize()
+            now = [t.view(torch.int16).clone() for t in (y, dx)] + [t.view(torch.int32).clone() for t in (dW1, dW2, dW3)] + \
+                  [torch.cat([v.view(-1) for v in list(sc.values()) + list(am.values())]).view(torch.int32).clone()]
+            if first is None:
+                first = now
+            else:
+                assert all(torch.equal(a, b) for a, b in zip(now, first)), f"just-in-time step, repetition {rep}"
+        s = sc["h"].clone()
+        B.fp8mlp_merge_weights(ctx, W1, W2, W3, s, B.SCALE_FROM_CURRENT_AMAX, sc, am)
+        B.fp8mlp_forward_merged(ctx, T, x, B.SCALE_FROM_CURRENT_AMAX, sc, am, y)
+        first = None
+        for rep in range(30):
+            y.fill_(float("nan"))
+            B.fp8mlp_forward_merged(ctx, T, x, B.SCALE_GIVEN, sc, None, y)
+            torch.cuda.synchronize()
+            now = y.view(torch.int16).clone()
+            if first is None:
+                first = now
+            else:
+                assert torch.equal(now, first), f"merged forward, repetition {rep}"
+        assert B.fp8mlp_status(ctx) == B.OK
+    finally:
+        B.fp8mlp_destroy(ctx)
