@@ -105,11 +105,13 @@ def test_gemm_plans_at_the_benchmark_shapes():
     g1, g2 = plan(B.GEMM_SWIGLU_FWD, T, f, d), plan(B.GEMM_BF16_OUT, T, d, f)
     assert (g1["cta_pairs"], g1["tile_rows"], g1["tile_cols"], g1["m_tiles"], g1["n_tiles"], g1["k_stages"]) == (1, 256, 128, 64, 86, 32)
     assert (g2["tile_cols"], g2["n_tiles"], g2["k_stages"], g2["split_k"], g2["staged_stores"]) == (512, 8, 86, 1, 1)
-    # rasterisation: bands along the smaller operand, cut so that a band's slice stays under 46 MB
+    # rasterisation: bands along the smaller operand, the whole of it while it is under 96 MiB
     assert (g2["band_along_n"], g2["band_tiles"]) == (1, 8)                                     # all of W3' (45 MB)
     w3, d1, w12 = plan(B.GEMM_F32_OUT, f, d, T), plan(B.GEMM_BF16_OUT, T, d, 2 * f), plan(B.GEMM_F32_OUT, d, 2 * f, T)
-    assert (w3["band_along_n"], w3["band_tiles"]) == (1, 8) and (d1["band_along_n"], d1["band_tiles"]) == (1, 4)
-    assert (w12["band_along_n"], w12["band_tiles"]) == (0, 8) and w12["work_items"] == 16 * 86 and w12["staged_stores"] == 0
+    assert (w3["band_along_n"], w3["band_tiles"]) == (1, 16) and (d1["band_along_n"], d1["band_tiles"]) == (1, 8)
+    assert (w12["band_along_n"], w12["band_tiles"]) == (0, 16) and w12["work_items"] == 16 * 86 and w12["staged_stores"] == 0
+    big = plan(B.GEMM_BF16_OUT, 8192, 8192, 2 * 28672)                                           # 70B input gradient: W12 is 470 MB
+    assert big["band_along_n"] == 0 or big["band_tiles"] < big["n_tiles"]
     assert (g1["band_along_n"], g1["band_tiles"]) == (0, 16)                                     # fused epilogues: 16 row tiles
     # T = 512: 32 tiles for 74 CTA pairs -> the long contractions are split in two; the weight gradients (4 stages of
     # work per tile) stage their output; without a context's workspace nothing is split
