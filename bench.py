@@ -37,7 +37,7 @@ FP8_OVER_BF16 = 2.0          # nominal dense tensor-core ratio (4.5 vs 2.25 PFLO
 NOMINAL_FP8_TFLOPS = 4500.0
 # DRAM bytes per launch of the dominant kernel (gate/up GEMM + SwiGLU epilogue) measured by ncu
 # (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None until captured.
-NCU_TRAFFIC_BYTES = {"7b": 446_591_000 + 864_400_640}     # profiles/gemm_kernels_7b.txt, GEMM-1 launch (read + write)
+NCU_TRAFFIC_BYTES = {"7b": 468_702_000 + 866_461_184}     # profiles/gemm_kernels_7b.txt, GEMM-1 launch (read + write)
 
 
 def flops_step(T, d, f):
